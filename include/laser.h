@@ -1,0 +1,169 @@
+/*
+ * laser.h -- C ABI of the LASER routing library for NVIDIA B200 (sm_100a).
+ *
+ * LASER (Load- and Score-based Expert Routing) is an inference-time router for
+ * Mixture-of-Experts layers.  For every token, in row order, this library computes
+ *   1. the gate logits  x = h . W_g^T (+ bias)            [Introduction: gating network]
+ *   2. the softmax scores s over all E experts             [The Method, Problem formulation]
+ *   3. the top-k mass M_k and the test M_k >= eps_high     [The Method, Expansion rule]
+ *   4. the candidate pool {s_i >= t_fix * s_max} united with the top-k, trimmed to the
+ *      c best                                              [Algorithm 1; Final assignment]
+ *   5. the k candidates with the smallest current load, ties by score
+ *                                                          [Algorithm 1, StableSortByLoad]
+ *   6. the load update L[e] += 1 for the k chosen experts, before the next token
+ *   7. combine weights, the per-expert dispatch (counts, offsets, permuted pair ids) and
+ *      per-device-bin load sums                            [Motivation: placement, N_g]
+ *
+ * General rules for every entry point
+ *   - Pointers are DEVICE pointers unless the parameter is documented as host.
+ *   - The caller owns every buffer; the library keeps no state between calls.
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*); the call
+ *     returns without synchronising, except laser_route_host, which synchronises the stream
+ *     before returning.
+ *   - Return value: LASER_OK (0) or a negative status.  On a validation error nothing is
+ *     launched and no output is touched.
+ *   - Conditions only visible on the device are OR-ed into *status_word (device int32,
+ *     may be NULL): LASER_DEV_LOAD_OVERFLOW.
+ */
+#ifndef LASER_H_
+#define LASER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  LASER_OK = 0,
+  LASER_ERR_INVALID_ARG = -1,      /* NULL where a buffer is required, or a size out of range */
+  LASER_ERR_UNSUPPORTED = -2,      /* a documented but unimplemented mode */
+  LASER_ERR_WORKSPACE_TOO_SMALL = -3,
+  LASER_ERR_MISALIGNED = -4,       /* hidden / W_g base or row stride not 16-byte aligned */
+  LASER_ERR_CUDA = -5              /* a CUDA runtime call failed (launch error) */
+};
+
+enum { LASER_DEV_LOAD_OVERFLOW = 1 }; /* bit in *status_word: a load counter passed 2^31-1 */
+
+enum { LASER_MAX_EXPERTS = 256 };
+
+/*
+ * Parameters of one routing call (host struct, read during the call only).
+ *
+ *   T            tokens (rows of hidden), >= 0
+ *   d            hidden size, > 0, multiple of 8
+ *   E            routed experts n, 1..LASER_MAX_EXPERTS
+ *   k            experts activated per token, 1 <= k <= c
+ *   c            trimming size of Algorithm 1, k <= c <= E
+ *   eps_high     dominance cutoff; the paper's domain is (0,1).  0 gives vanilla top-k for
+ *                every token, a value above 1 expands every token.
+ *   t_fix        pool threshold relative to the best score; paper's domain (0,1], 0 allowed
+ *                (pool = the c best).  eps_high > 1, t_fix = 0, c = E is load-only routing.
+ *   trim_mode    0 = TOP (keep the c best).  1 = RANDOM is not implemented
+ *                (LASER_ERR_UNSUPPORTED).
+ *   update_granularity  1 = loads are updated after every token (the only mode).
+ *   renormalize  1: combine weights are divided by their sum over the k chosen experts;
+ *                0: raw softmax scores.
+ *   n_bins       number of device bins B >= 1 (only used when bin_loads != NULL)
+ *   ld_hidden, ld_w   row strides of hidden and W_g in elements (>= d, multiple of 8)
+ */
+typedef struct laser_params {
+  int32_t T, d, E, k, c;
+  float eps_high;
+  float t_fix;
+  int32_t trim_mode;
+  int32_t update_granularity;
+  int32_t renormalize;
+  int32_t n_bins;
+  int64_t ld_hidden, ld_w;
+  uint64_t seed; /* reserved for RANDOM trimming */
+} laser_params;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int laser_version(void);
+
+/* Static description of a status code.  Never NULL. */
+const char* laser_strerror(int status);
+
+/*
+ * Scratch bytes one layer of laser_route needs for these parameters (candidate records of
+ * stage 4 and block histograms of stage 7).  p and bytes are host pointers.
+ */
+int laser_workspace_bytes(const laser_params* p, size_t* bytes);
+
+/*
+ * Route one MoE layer (stages 1-7 above).
+ *
+ *   hidden      [T, ld_hidden] bf16, row-major, 16-byte aligned
+ *   w_g         [E, ld_w]      bf16, one row per expert, 16-byte aligned
+ *   bias        [E] fp32 added to the logits, or NULL
+ *   loads       [E] int32, in/out: L on entry, L + per-call counts on return
+ *   expert_to_bin [E] int32 in [0, n_bins), or NULL for contiguous e / ceil(E / n_bins)
+ *   bin_loads   [n_bins] int32 in/out, or NULL to skip bin accounting
+ *   p           host
+ *   expert_ids  [T, k] int32 out.  Top-k branch: descending score.  Expanded branch:
+ *               ascending (load, score rank).
+ *   weights     [T, k] fp32 out, weights[t,j] belongs to expert_ids[t,j]
+ *   offsets     [E+1] int32 out, exclusive prefix of this call's per-expert counts
+ *   perm        [T*k] int32 out: pair ids t*k+j grouped by expert, ascending within an expert
+ *   logits_out  [T, E] fp32 out, or NULL.  Never changes a decision.
+ *   status_word device int32 or NULL (bits are OR-ed in, never cleared)
+ *   workspace   device scratch of at least laser_workspace_bytes(), 256-byte aligned
+ */
+int laser_route(const void* hidden, const void* w_g, const float* bias,
+                int32_t* loads, const int32_t* expert_to_bin, int32_t* bin_loads,
+                const laser_params* p,
+                int32_t* expert_ids, float* weights, int32_t* offsets, int32_t* perm,
+                float* logits_out, int32_t* status_word,
+                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Route n_layers independent MoE layers that share one shape in one call.  Layer l uses
+ * element l of every array below; each layer has its own W_g, bias, loads and outputs, and
+ * the result equals n_layers calls of laser_route.
+ *
+ *   hidden [n_layers, T, ld_hidden]   w_g [n_layers, E, ld_w]   bias [n_layers, E] or NULL
+ *   loads [n_layers, E]               bin_loads [n_layers, n_bins] or NULL
+ *   expert_to_bin [E] shared by all layers, or NULL
+ *   eps_high_per_layer, t_fix_per_layer: HOST arrays [n_layers] or NULL (use p's value)
+ *   expert_ids [n_layers, T, k]  weights [n_layers, T, k]  offsets [n_layers, E+1]
+ *   perm [n_layers, T*k]         logits_out [n_layers, T, E] or NULL
+ *   workspace: n_layers * laser_workspace_bytes() bytes
+ */
+int laser_route_layers(int32_t n_layers,
+                       const void* hidden, const void* w_g, const float* bias,
+                       int32_t* loads, const int32_t* expert_to_bin, int32_t* bin_loads,
+                       const laser_params* p,
+                       const float* eps_high_per_layer, const float* t_fix_per_layer,
+                       int32_t* expert_ids, float* weights, int32_t* offsets, int32_t* perm,
+                       float* logits_out, int32_t* status_word,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Device bytes laser_route_host needs in its arena for n_layers layers (inputs, outputs and
+ * workspace).  p and bytes are host pointers.
+ */
+int laser_host_arena_bytes(int32_t n_layers, const laser_params* p, size_t* bytes);
+
+/*
+ * laser_route_layers with HOST buffers: copies the inputs to the device arena, routes,
+ * copies expert_ids, weights, offsets, perm, loads and bin_loads back, and synchronises the
+ * stream.  Every array argument has the layout of laser_route_layers but lives in host
+ * memory (pinned memory makes the copies asynchronous); arena is device memory of at least
+ * laser_host_arena_bytes(), 256-byte aligned.  loads / bin_loads are in/out on the host.
+ * status_out (host int32, may be NULL) receives the device status word.
+ */
+int laser_route_host(int32_t n_layers,
+                     const void* hidden, const void* w_g, const float* bias,
+                     int32_t* loads, const int32_t* expert_to_bin, int32_t* bin_loads,
+                     const laser_params* p,
+                     const float* eps_high_per_layer, const float* t_fix_per_layer,
+                     int32_t* expert_ids, float* weights, int32_t* offsets, int32_t* perm,
+                     int32_t* status_out,
+                     void* arena, size_t arena_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LASER_H_ */

@@ -1,0 +1,93 @@
+"""Pure-Python restatements used to cross-check the C oracle on small inputs.
+
+TEST INFRASTRUCTURE, not a product path.  Three independent pieces:
+
+* ``alg1_token``   -- Algorithm 1 of the paper taken literally: a candidate *set* built by
+  thresholding all n scores, united with the top-k, trimmed to the c* highest-scoring, then
+  a stable sort by load with score as tie-break.
+* ``brute_force_token`` -- the selection step by exhaustive search: among all k-subsets of
+  the candidate set, the one whose sorted (load, score-rank) key vector is smallest.
+* ``imbalance`` / ``max_violation`` -- the imbalance factor of Motivation and MV of
+  Evaluation/Metrics.
+"""
+from __future__ import annotations
+
+import itertools
+
+import numpy as np
+
+
+def score_order(s, x=None):
+    """Indices by score descending; ties by logit descending (if given), then index."""
+    n = len(s)
+    if x is None:
+        return sorted(range(n), key=lambda i: (-float(s[i]), i))
+    return sorted(range(n), key=lambda i: (-float(s[i]), -float(x[i]), i))
+
+
+def alg1_token(s, L, k, c, eps_high, t_fix, x=None):
+    """Algorithm 1 (TOP trimming) for one token.  s: fp32 scores, L: integer loads.
+
+    Returns (A as a list in the order the sorted candidate list yields, expanded flag,
+    c*).  All comparisons on scores are made in fp32, as the scores are given.
+    """
+    s = np.asarray(s, np.float32)
+    n = len(s)
+    order = score_order(s, x)
+    Mk = np.float32(s[order[0]])
+    for j in range(1, k):
+        Mk = np.float32(Mk + s[order[j]])
+    if Mk >= np.float32(eps_high):
+        return list(order[:k]), False, 0
+    t = np.float32(np.float32(t_fix) * s[order[0]])
+    pool = {i for i in range(n) if s[i] >= t} | set(order[:k])
+    m = len(pool)
+    c_star = min(c, m)
+    by_score = [i for i in order if i in pool]
+    cand = by_score[:c_star]
+    # stable sort by load; cand is already in descending score order, so stability
+    # realises "ties broken by score, descending".
+    cand_sorted = sorted(cand, key=lambda i: int(L[i]))
+    return cand_sorted[:k], True, c_star
+
+
+def alg1_sequence(S, loads, k, c, eps_high, t_fix, X=None):
+    """Route the rows of S in order, adding one to the load of each chosen expert after
+    every token.  Returns (ids [T][k], final loads, expanded flags)."""
+    L = [int(v) for v in loads]
+    ids, flags = [], []
+    for t in range(len(S)):
+        A, expanded, _ = alg1_token(S[t], L, k, c, eps_high, t_fix, None if X is None else X[t])
+        for e in A:
+            L[e] += 1
+        ids.append(A)
+        flags.append(expanded)
+    return ids, L, flags
+
+
+def brute_force_token(cand_in_rank_order, L, k):
+    """Best k-subset of the candidates by exhaustive search.
+
+    A candidate's key is (load, score rank).  A subset is scored by its keys sorted
+    ascending; the lexicographically smallest vector wins.  Returned in key order.
+    """
+    keyed = [(int(L[e]), r, e) for r, e in enumerate(cand_in_rank_order)]
+    best = None
+    for sub in itertools.combinations(keyed, k):
+        vec = sorted(sub)
+        if best is None or vec < best:
+            best = vec
+    return [e for (_, _, e) in best]
+
+
+def imbalance(counts) -> float:
+    """I = max_e N_e / mean_e N_e  (Motivation, expert imbalance of one layer and batch)."""
+    counts = np.asarray(counts, np.float64)
+    mean = counts.mean()
+    return float(counts.max() / mean) if mean > 0 else 1.0
+
+
+def max_violation(counts) -> float:
+    """MV, read as how far the most loaded expert exceeds the average, relative to it:
+    max/mean - 1 (zero for perfect balance, as the load-only baseline attains)."""
+    return imbalance(counts) - 1.0

@@ -1,0 +1,270 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (CPU only)."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import alg1_literal as lit
+from paper_2510_03293_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rand_logits(rng, T, E, spread=2.0):
+    scale = np.exp(rng.uniform(np.log(0.1), np.log(3.0), size=(T, 1)))
+    return (rng.standard_normal((T, E)) * scale * spread).astype(np.float32)
+
+
+# ---------------------------------------------------------------- exp / softmax
+def test_exp32_matches_exp_and_is_exact_at_zero():
+    assert oracle.exp32(0.0) == np.float32(1.0)
+    assert oracle.exp32(-81.0) == np.float32(0.0)
+    ys = np.concatenate([-np.logspace(-6, math.log10(79.0), 4000), -np.linspace(0, 2, 3001)])
+    for y in ys.astype(np.float32):
+        got = float(oracle.exp32(y))
+        want = math.exp(float(y))
+        assert abs(got - want) <= 3e-7 * want, (y, got, want)
+
+
+def test_exp32_monotone_on_dense_grid():
+    # the prefix form of the candidate pool assumes scores do not invert the logit order
+    ys = -np.linspace(0.0, 30.0, 200001).astype(np.float32)
+    vals = np.array([oracle.exp32(y) for y in ys])
+    assert np.all(np.diff(vals) <= 0)
+
+
+@pytest.mark.parametrize("E", [1, 2, 5, 8, 13, 64, 256])
+def test_softmax_is_a_distribution_and_matches_fp64(E):
+    rng = np.random.default_rng(E)
+    x = rand_logits(rng, 64, E, spread=3.0)
+    s = oracle.softmax(x)
+    assert np.all(s >= 0)
+    assert np.max(np.abs(s.astype(np.float64).sum(1) - 1.0)) <= E * 2.0 ** -22
+    x64 = x.astype(np.float64)
+    ref = np.exp(x64 - x64.max(1, keepdims=True))
+    ref /= ref.sum(1, keepdims=True)
+    big = ref > 1e-30
+    # x - x_max is rounded to fp32 first: with |x| up to ~30 that alone is ~2e-6 relative
+    assert np.max(np.abs(s[big] - ref[big]) / ref[big]) <= 5e-6
+
+
+# ---------------------------------------------------------------- logits
+def test_logits_hand_example_and_fp64_matmul():
+    h = synth.f32_to_bf16_bits(np.array([[1.0, 2.0, 0.5, -4.0, 0, 0, 0, 0]], np.float32))
+    w = synth.f32_to_bf16_bits(np.array([[3.0, 4.0, 2.0, 1.0, 0, 0, 0, 0],
+                                         [0.5, -1.0, 8.0, 0.25, 0, 0, 0, 0]], np.float32))
+    x = oracle.logits(h, w, np.array([0.0, 10.0], np.float32))
+    assert x.tolist() == [[3 + 8 + 1 - 4, 0.5 - 2 + 4 - 1 + 10.0]]
+
+    hb, wb, bias = synth.make_layer(37, 264, 11, 0.02, 1.2, seed=3, stream=7)
+    x = oracle.logits(hb, wb, bias)
+    ref = synth.bf16_bits_to_f32(hb).astype(np.float64) @ synth.bf16_bits_to_f32(wb).astype(np.float64).T
+    ref = ref.astype(np.float32) + bias
+    assert np.max(np.abs(x - ref)) <= 1e-6
+    # a transposed or mis-strided operand would not survive a non-square case
+    assert x.shape == (37, 11)
+
+
+# ---------------------------------------------------------------- reductions to top-k
+@pytest.mark.parametrize("E,k", [(8, 2), (64, 6), (5, 1), (6, 6)])
+def test_eps_zero_is_vanilla_topk(E, k):
+    rng = np.random.default_rng(10 * E + k)
+    x = rand_logits(rng, 300, E)
+    x[5] = x[5, 0]                      # all-equal row: ties go to the lower index
+    x[6, 1] = x[6, 3]
+    ids, w, L, cs = oracle.route(x, rng.integers(0, 50, E), k, min(E, k + 2), 0.0, 0.5)
+    assert np.all(cs == 0)
+    assert np.array_equal(ids, oracle.topk(x, k))
+    # textbook top-k through a library sort (stable, on negated logits)
+    ref = np.argsort(-x.astype(np.float64), axis=1, kind="stable")[:, :k]
+    assert np.array_equal(ids, ref)
+
+
+@pytest.mark.parametrize("E,k", [(8, 2), (64, 6)])
+def test_c_equal_k_is_topk_as_sets(E, k):
+    rng = np.random.default_rng(E)
+    x = rand_logits(rng, 400, E)
+    loads = rng.integers(0, 1000, E)
+    ids, _, _, cs = oracle.route(x, loads, k, k, 2.0, 0.3)     # every token expands
+    assert np.all(cs == k)
+    top = oracle.topk(x, k)
+    assert np.array_equal(np.sort(ids, 1), np.sort(top, 1))
+
+
+# ---------------------------------------------------------------- pool and selection
+def test_pool_closed_form_and_selection_properties():
+    rng = np.random.default_rng(77)
+    E, k, c, eps, tfix = 16, 3, 7, 0.9, 0.4
+    x = rand_logits(rng, 600, E, spread=1.0)
+    loads0 = rng.integers(0, 6, E).astype(np.int32)
+    ids, w, L, cs = oracle.route(x, loads0, k, c, eps, tfix)
+    s = oracle.softmax(x)
+    cur = loads0.copy()
+    gap = math.log(1.0 / tfix)
+    n_expanded = 0
+    for t in range(x.shape[0]):
+        order = np.argsort(-x[t].astype(np.float64), kind="stable")
+        A = ids[t]
+        assert len(set(A.tolist())) == k
+        if cs[t] > 0:
+            n_expanded += 1
+            # closed form on the logits: s_i >= t_fix * s_max  <=>  x_max - x_i <= ln(1/t_fix)
+            d = float(x[t, order[0]]) - x[t].astype(np.float64)
+            if np.min(np.abs(d - gap)) > 1e-4:
+                m_all = int(np.sum(d <= gap))
+                assert cs[t] == min(c, max(k, m_all))
+            cand = order[:cs[t]]
+            assert set(A.tolist()) <= set(cand.tolist())
+            rank = {int(e): j for j, e in enumerate(cand)}
+            keys = [(int(cur[e]), rank[int(e)]) for e in A]
+            assert keys == sorted(keys)                      # listed in increasing key order
+            rest = [(int(cur[e]), rank[int(e)]) for e in cand if e not in A]
+            if rest:
+                assert max(keys) < min(rest)                 # least loaded within the pool
+        else:
+            assert A.tolist() == order[:k].tolist()
+        cur[A] += 1
+    assert 50 < n_expanded < 590                             # both branches exercised
+    assert np.array_equal(cur, L)
+    assert int((L - loads0).sum()) == x.shape[0] * k
+    # weights belong to their ids and renormalise to one
+    assert np.max(np.abs(w.astype(np.float64).sum(1) - 1.0)) <= 4 * 2.0 ** -23 * k
+    ids2, w2, _, _ = oracle.route(x, loads0, k, c, eps, tfix, renormalize=False)
+    assert np.array_equal(ids, ids2)
+    assert np.array_equal(w2, np.take_along_axis(s, ids2, 1))
+
+
+def test_topk_always_in_pool_with_tfix_one():
+    rng = np.random.default_rng(5)
+    x = rand_logits(rng, 200, 8)
+    ids, _, _, cs = oracle.route(x, np.zeros(8), 2, 8, 2.0, 1.0)
+    assert np.all(cs >= 2)
+    assert np.array_equal(np.sort(ids, 1), np.sort(oracle.topk(x, 2), 1))
+
+
+def test_load_only_gives_perfect_balance():
+    # eps_high > 1, t_fix = 0, c = n ignores the scores: after every token max-min <= 1
+    rng = np.random.default_rng(9)
+    E, k, T = 8, 2, 400
+    x = rand_logits(rng, T, E)
+    L = np.zeros(E, np.int32)
+    for t in range(T):
+        _, _, L, _ = oracle.route(x[t:t + 1], L, k, E, 2.0, 0.0)
+        assert L.max() - L.min() <= 1
+    assert lit.imbalance(L) == 1.0 and lit.max_violation(L) == 0.0
+    _, _, L2, _ = oracle.route(x, np.zeros(E), k, E, 2.0, 0.0)
+    assert np.array_equal(L, L2)                             # split calls == one call
+
+
+def test_split_call_equivalence():
+    rng = np.random.default_rng(21)
+    x = rand_logits(rng, 301, 64)
+    L0 = rng.integers(0, 9, 64)
+    ids, w, L, cs = oracle.route(x, L0, 6, 8, 0.5, 0.7)
+    ida, wa, La, _ = oracle.route(x[:150], L0, 6, 8, 0.5, 0.7)
+    idb, wb, Lb, _ = oracle.route(x[150:], La, 6, 8, 0.5, 0.7)
+    assert np.array_equal(ids, np.vstack([ida, idb]))
+    assert np.array_equal(w, np.vstack([wa, wb]))
+    assert np.array_equal(L, Lb)
+
+
+# ---------------------------------------------------------------- literal Algorithm 1, brute force
+@pytest.mark.parametrize("E,k,c,eps,tfix", [(8, 2, 4, 0.64, 0.6), (16, 3, 16, 0.5, 0.3),
+                                             (64, 6, 8, 0.4, 0.8), (5, 2, 5, 0.8, 0.5)])
+def test_literal_algorithm_1_agrees(E, k, c, eps, tfix):
+    rng = np.random.default_rng(E * 100 + c)
+    x = rand_logits(rng, 250, E, spread=1.0)
+    L0 = rng.integers(0, 4, E)
+    ids, _, L, cs = oracle.route(x, L0, k, c, eps, tfix)
+    S = oracle.softmax(x)
+    ids_lit, L_lit, flags = lit.alg1_sequence(S, L0, k, c, eps, tfix, X=x)
+    assert [list(map(int, r)) for r in ids] == [list(map(int, r)) for r in ids_lit]
+    assert list(map(int, L)) == L_lit
+    assert flags == [bool(v) for v in cs > 0]
+
+
+def test_brute_force_small():
+    # every load vector in {0,1,2}^n for n = 4, and random ones for n = 6, T <= 8
+    rng = np.random.default_rng(2)
+    n, k = 4, 2
+    x = rand_logits(rng, 3, n, spread=0.3)
+    for loads in itertools.product(range(3), repeat=n):
+        ids, _, _, cs = oracle.route(x, np.array(loads), k, n, 2.0, 0.2)
+        for t in range(x.shape[0]):
+            cur = np.array(loads)
+            for u in range(t):
+                cur[ids[u]] += 1
+            order = np.argsort(-x[t].astype(np.float64), kind="stable")[:cs[t]]
+            assert ids[t].tolist() == lit.brute_force_token(order.tolist(), cur, k)
+    n, k = 6, 3
+    for trial in range(40):
+        x = rand_logits(rng, 8, n, spread=0.5)
+        loads = rng.integers(0, 3, n)
+        ids, _, _, cs = oracle.route(x, loads, k, 5, 2.0, 0.5)
+        cur = loads.copy()
+        for t in range(8):
+            order = np.argsort(-x[t].astype(np.float64), kind="stable")[:cs[t]]
+            assert ids[t].tolist() == lit.brute_force_token(order.tolist(), cur, k)
+            cur[ids[t]] += 1
+
+
+def test_overview_figure_scenario():
+    rows = [l for l in open(os.path.join(GOLDEN, "figure_overview_scenario.txt"))
+            if l.strip() and not l.startswith("#")]
+    for line in rows:
+        s_txt, l_txt, a_txt = line.split("|")
+        s = np.array(s_txt.split(), np.float64)
+        loads = np.array(l_txt.split(), np.int32)
+        want = set(map(int, a_txt.split()))
+        x = np.log(s).astype(np.float32)[None, :]
+        ids, _, _, _ = oracle.route(x, loads, 2, 5, 0.8, 0.5)
+        assert set(ids[0].tolist()) == want
+        A, _, _ = lit.alg1_token(s.astype(np.float32), loads, 2, 5, 0.8, 0.5)
+        assert set(A) == want
+
+
+# ---------------------------------------------------------------- dispatch, bins, parameters
+def test_dispatch_properties_and_library_sort():
+    rng = np.random.default_rng(4)
+    T, k, E = 513, 3, 10
+    ids = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
+    offsets, perm = oracle.dispatch(ids, E)
+    flat = ids.reshape(-1)
+    assert offsets[0] == 0 and offsets[E] == T * k
+    assert np.array_equal(np.diff(offsets), np.bincount(flat, minlength=E))
+    assert np.array_equal(np.sort(perm), np.arange(T * k))
+    assert np.all(np.diff(flat[perm]) >= 0)
+    assert np.array_equal(perm, np.argsort(flat, kind="stable"))
+    # an expert nobody chose keeps an empty segment
+    ids2 = np.where(ids == 4, 9, ids)
+    off2, _ = oracle.dispatch(np.sort(ids2, 1), E)
+    assert off2[5] == off2[4]
+
+
+def test_bins_sum_member_counts():
+    counts = np.arange(8, dtype=np.int32) + 1
+    e2b = synth.default_expert_to_bin(8, 4)
+    out = oracle.bins(counts, e2b, np.array([100, 0, 0, 0], np.int32))
+    assert out.tolist() == [100 + 1 + 2, 3 + 4, 5 + 6, 7 + 8]
+    assert int(out.sum()) - 100 == int(counts.sum())
+
+
+def test_workload_parameters_come_from_the_papers_table():
+    table = {}
+    for line in open(os.path.join(GOLDEN, "paper_thresholds.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        model, dataset, tfix, eps = [p.strip() for p in line.split("|")]
+        table[(model, dataset)] = (tuple(map(float, tfix.split("/"))), tuple(map(float, eps.split("/"))))
+    mix = table[("Mixtral-8x7B", "ARC Challenge")]
+    ds = table[("DeepSeek-MoE-16B-Chat", "MMLU")]
+    w = synth.WORKLOADS
+    assert w["mixtral"].eps_high == mix[1] and w["mixtral"].t_fix == mix[0][0]
+    assert w["tiny"].eps_high == (mix[1][1],)
+    assert w["deepseek"].eps_high == (ds[1][0],) and w["deepseek"].t_fix == ds[0][0]
+    assert w["stress"].t_fix == min(min(v[0]) for v in table.values())
+    assert [w["mixtral"].eps_for_layer(l) for l in (0, 10, 11, 21, 22, 31)] == \
+        [mix[1][0], mix[1][0], mix[1][1], mix[1][1], mix[1][2], mix[1][2]]
