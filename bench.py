@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of the LASER routing path: routed tokens/s for router + LASER + dispatch.
+
+A step is one pass of the whole path (router contraction, score epilogue, ordered load-aware
+selection, load update, dispatch, bin accounting) over every layer of the Mixtral-8x7B-shaped
+workload: 32 independent MoE layers x 16384 tokens, d=4096 bf16, E=8, k=2, loads reset per
+step.  Inputs are seeded synthetic tensors (4.3 GB of hidden states, larger than L2).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints one JSON line.  With --impl reference the CPU oracle is timed on the host cores on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "routed tokens/sec per B200 (router+LASER+dispatch)"
+UNIT = "tokens/s"
+
+
+def measured_peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def algorithmic_bytes_per_token(w) -> float:
+    """Bytes the method must move per token: the bf16 hidden row, k x (id, weight, perm entry)
+    and the amortised W_g."""
+    return 2.0 * w.d + 12.0 * w.k + 2.0 * w.E * w.d / w.T
+
+
+def workload_config(w, n_layers):
+    return {"workload": "%s: %d layers x T=%d, d=%d bf16, E=%d, k=%d, c=%d, %d bins" %
+            (w.name, n_layers, w.T, w.d, w.E, w.k, w.c, w.n_bins),
+            "tokens_per_step": n_layers * w.T, "t_fix": w.t_fix, "eps_high": list(w.eps_high),
+            "cache": "inputs (%.2f GB per step) exceed the 126 MB L2" %
+                     (2.0 * n_layers * w.T * w.d / 1e9)}
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_pass(oracle, np, layers_data, w, eps, tfix):
+    """The oracle's whole path on a list of (hidden_bits, wg_bits, bias) layers."""
+    from paper_2510_03293_b200 import synth
+
+    e2b = synth.default_expert_to_bin(w.E, w.n_bins)
+    t0 = time.perf_counter()
+    for l, (hb, wb, bias) in enumerate(layers_data):
+        oracle.route_full(hb, wb, bias, np.zeros(w.E, np.int32), e2b, np.zeros(w.n_bins, np.int32),
+                          w.k, w.c, eps[l], tfix[l], bool(w.renormalize))
+    return time.perf_counter() - t0
+
+
+def run_reference(args, w):
+    import numpy as np
+
+    import oracle
+    from paper_2510_03293_b200 import synth
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    oracle.build()
+    n_sample = min(w.layers, args.ref_layers)
+    data = [synth.make_workload_layer(w, l) for l in range(n_sample)]
+    eps = [w.eps_for_layer(l) for l in range(n_sample)]
+    tfix = [w.t_fix] * n_sample
+    for _ in range(args.warmup):
+        oracle_pass(oracle, np, data[:1], w, eps, tfix)
+    times = [oracle_pass(oracle, np, data, w, eps, tfix) for _ in range(args.steps)]
+    sec = sum(times) / len(times)
+    value = n_sample * w.T / sec
+    cores = len(os.sched_getaffinity(0))
+    sample = "%d of %d layers per step (%d tokens)" % (n_sample, w.layers, n_sample * w.T)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(w, n_sample),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=fd,
+                stderr=subprocess.DEVNULL)
+            os.close(fd)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.strip().split(", ") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, reasons, mx = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx = float(r[2])
+            except ValueError:
+                continue
+            for name, v in zip(names, r[5:9]):
+                if v.strip().lower() == "active":
+                    reasons.add(name)
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=mx, reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_gpu(args, w):
+    import numpy as np
+    import torch
+
+    from paper_2510_03293_b200 import laser, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    L = w.layers if args.layers is None else args.layers
+    data = synth.make_workload_torch(w, dev, seed=args.seed + rank, layers=L)
+    p = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize, w.n_bins)
+    loads = torch.zeros((L, w.E), dtype=torch.int32, device=dev)
+    bins = torch.zeros((L, w.n_bins), dtype=torch.int32, device=dev)
+    ws = torch.empty((laser.workspace_bytes(p) * L,), dtype=torch.uint8, device=dev)
+    out = None
+
+    def step(events=None):
+        nonlocal out
+        loads.zero_(); bins.zero_()
+        out = laser.route_layers(data["hidden"], data["w_g"], data["bias"], loads, p,
+                                 bin_loads=bins, eps_high=data["eps_high"], t_fix=data["t_fix"],
+                                 out=out, workspace=ws, stage_events=events)
+
+    def new_events(n):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in evs:
+            e.record()
+        return evs
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    stage = [new_events(4) for _ in range(args.steps)]
+    t_begin, t_end = new_events(2)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    t_begin.record()
+    for i in range(args.steps):
+        step(stage[i])
+    t_end.record()
+    barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    tokens = L * w.T
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    k1 = sum(ev[0].elapsed_time(ev[1]) for ev in stage) / args.steps
+    k2 = sum(ev[1].elapsed_time(ev[2]) for ev in stage) / args.steps
+    k3 = sum(ev[2].elapsed_time(ev[3]) for ev in stage) / args.steps
+    peak, peak_kind = measured_peak_hbm()
+    bytes_per_launch = algorithmic_bytes_per_token(w) * tokens
+    achieved = bytes_per_launch / (k1 * 1e-3) / 1e9
+    path_gbs = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
+
+    status = int(out.status.item())
+    counts = (out.offsets[:, 1:] - out.offsets[:, :-1]).double()
+    imb = float((counts.max(1).values / counts.mean(1)).mean().item())
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate and scores",
+        "data": "synthetic", "config": workload_config(w, L),
+        "roofline": {"bound": "hbm", "kernel": "k1_router_mma (contraction + score epilogue)",
+                     "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None,
+                     "bytes_per_launch": bytes_per_launch},
+        "path": {"k1_ms": k1, "k2_ms": k2, "k3_ms": k3, "path_gbs": path_gbs,
+                 "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
+        "routing": {"mean_imbalance_max_over_mean": imb, "status_word": status},
+        "gpu_launches": 6 * ((L + 63) // 64) * args.steps,
+        "clocks": clocks,
+    }
+
+    # end to end through the host-buffer entry point: H2D of the inputs, D2H of the results
+    if world == 1 or rank == 0:
+        result["e2e"] = e2e_host(args, w, L, data, p, laser, torch, dev)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(args, w, L, data, np)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result))
+
+
+def e2e_host(args, w, L, data, p, laser, torch, dev):
+    h_hidden = data["hidden"].cpu().pin_memory()
+    h_wg = data["w_g"].cpu().pin_memory()
+    h_bias = data["bias"].cpu().pin_memory()
+    h_loads = torch.zeros((L, w.E), dtype=torch.int32).pin_memory()
+    h_bins = torch.zeros((L, w.n_bins), dtype=torch.int32).pin_memory()
+    arena = torch.empty((laser.host_arena_bytes(L, p),), dtype=torch.uint8, device=dev)
+    outs = None
+    times = []
+    n = max(1, min(args.steps, args.e2e_steps))
+    for i in range(n + 1):
+        h_loads.zero_(); h_bins.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        outs = laser.route_host(h_hidden, h_wg, h_bias, h_loads, p, arena, bin_loads=h_bins,
+                                eps_high=data["eps_high"], t_fix=data["t_fix"], out=outs)
+        if i > 0:
+            times.append(time.perf_counter() - t0)
+    sec = sum(times) / len(times)
+    h2d = sum(t.numel() * t.element_size() for t in (h_hidden, h_wg, h_bias, h_loads, h_bins))
+    d2h = sum(t.numel() * t.element_size() for t in outs) + \
+        sum(t.numel() * t.element_size() for t in (h_loads, h_bins))
+    return {"value": L * w.T / sec, "unit": UNIT, "ms_per_step": sec * 1e3,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n}
+
+
+def cpu_baseline(args, w, L, data, np):
+    import oracle
+
+    oracle.build()
+    n_sample = min(L, args.ref_layers)
+    layers_data = []
+    for l in range(n_sample):
+        hb = data["hidden"][l].view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+        wb = data["w_g"][l].view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+        layers_data.append((hb, wb, data["bias"][l].cpu().numpy()))
+    sec = oracle_pass(oracle, np, layers_data, w, data["eps_high"], data["t_fix"])
+    return {"value": n_sample * w.T / sec, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+            "kind": "oracle", "seconds": sec,
+            "sample": "%d of %d layers (%d tokens), fp64 contraction with OpenMP over tokens, "
+                      "ordered scan on one core" % (n_sample, L, n_sample * w.T)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="laser", choices=["laser", "reference"])
+    ap.add_argument("--workload", default="mixtral")
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-layers", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2510_03293_b200 import synth
+
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()

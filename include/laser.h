@@ -141,6 +141,25 @@ int laser_route_layers(int32_t n_layers,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * laser_route_layers that also records CUDA events between its stages, so that a caller can
+ * time the router contraction (stage 1-4), the ordered selection (5-6) and the dispatch (7)
+ * separately.  stage_events is a HOST array of four cudaEvent_t handles (entries may be NULL),
+ * recorded on cuda_stream: [0] before the first kernel, [1] after the contraction + score
+ * epilogue, [2] after the selection, load update and combine weights, [3] after the dispatch.
+ * With more than 64 layers the stages run once per group of 64 and the events keep the last
+ * group's marks.  stage_events == NULL makes this identical to laser_route_layers.
+ */
+int laser_route_layers_profiled(int32_t n_layers,
+                                const void* hidden, const void* w_g, const float* bias,
+                                int32_t* loads, const int32_t* expert_to_bin, int32_t* bin_loads,
+                                const laser_params* p,
+                                const float* eps_high_per_layer, const float* t_fix_per_layer,
+                                int32_t* expert_ids, float* weights, int32_t* offsets,
+                                int32_t* perm, float* logits_out, int32_t* status_word,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                void* const* stage_events);
+
+/*
  * Device bytes laser_route_host needs in its arena for n_layers layers (inputs, outputs and
  * workspace).  p and bytes are host pointers.
  */

@@ -1,0 +1,229 @@
+// K1: router contraction x = h.W_g^T + b fused with the per-token score epilogue
+// (softmax, ranking of the c best, top-k mass test, candidate count c*).
+//
+// Streaming design for small/medium E: each warp owns MT*16 token rows and walks the hidden
+// dimension in chunks of 32 elements.  A thread reads 16 contiguous bytes of a row straight
+// from global memory into the A fragment of two m16n8k16 bf16 MMAs (the contraction index is
+// permuted identically for A and B, which a dot product allows), so hidden states go
+// HBM -> registers -> tensor core with no shared-memory staging.  W_g is small and stays in
+// L1/L2.  Accumulators are fp32.
+#pragma once
+#include "laser_common.cuh"
+
+namespace laser {
+
+__device__ __forceinline__ uint4 ldg_stream(const uint16_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1,
+                                               uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+      "{%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Per-token epilogue run by one thread on a row of fp32 logits in shared memory.
+//   ranking pi by (logit desc, index asc); e_i = exp32(x_i - x_max);
+//   Z = eight interleaved running sums combined pairwise; s = e / Z;
+//   M_k = s_pi(0) + ... + s_pi(k-1) left to right; top-k branch iff M_k >= eps_high;
+//   otherwise c* = max(k, #{j < c : s_pi(j) >= t_fix * s_pi(0)}).
+// Writes the record (c*, ranked ids, ranked scores) for the load-aware scan and, for every
+// token, the top-k ids and weights (final for the top-k branch, overwritten otherwise).
+__device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int E, int k, int c,
+                                               float eps_high, float t_fix, int renorm,
+                                               uint16_t* cstar, uint8_t* cand_ids,
+                                               float* cand_scores, int32_t* expert_ids,
+                                               float* weights) {
+  float xmax = x[0];
+  for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, x[i]);
+
+  float a[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) a[j] = 0.0f;
+  for (int i0 = 0; i0 < E; i0 += 8) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (i0 + j < E) a[j] = __fadd_rn(a[j], exp32(__fsub_rn(x[i0 + j], xmax)));
+    }
+  }
+  const float Z = __fadd_rn(__fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3])),
+                            __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7])));
+
+  float prev_x = __int_as_float(0x7f800000);  // +inf
+  int prev_i = -1;
+  float Mk = 0.0f, thr = 0.0f;
+  int mprime = 0;
+  for (int r = 0; r < c; ++r) {
+    float bx = 0.0f;
+    int bi = -1;
+    for (int i = 0; i < E; ++i) {
+      const float xi = x[i];
+      const bool after_prev = (xi < prev_x) || (xi == prev_x && i > prev_i);
+      if (after_prev && (bi < 0 || xi > bx)) { bx = xi; bi = i; }
+    }
+    const float s = __fdiv_rn(exp32(__fsub_rn(bx, xmax)), Z);
+    if (r == 0) { thr = __fmul_rn(t_fix, s); Mk = s; }
+    else if (r < k) Mk = __fadd_rn(Mk, s);
+    if (s >= thr) ++mprime;
+    cand_ids[r] = (uint8_t)bi;
+    cand_scores[r] = s;
+    if (r < k) { expert_ids[r] = bi; weights[r] = s; }
+    prev_x = bx;
+    prev_i = bi;
+  }
+  const bool top_k_branch = (Mk >= eps_high);
+  *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
+  if (top_k_branch && renorm) {
+    for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
+  }
+}
+
+// NT: 8-expert column tiles (E padded up to NT*8).  MT: 16-row tiles per warp.
+// KU: chunks of 32 hidden elements issued per loop trip.
+template <int NT, int MT, int KU>
+__global__ void __launch_bounds__(128) k1_router_mma(const RouteArgs A) {
+  extern __shared__ float smem_tile[];
+  constexpr int ROWS = MT * 16;
+  constexpr int EP = NT * 8;
+  constexpr int LDS = EP + 1;
+
+  const int layer = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q = lane & 3;
+  const int T = A.T, d = A.d, E = A.E;
+  const long long tok0 = ((long long)blockIdx.x * 4 + warp) * ROWS;
+  if (tok0 >= T) return;
+
+  const uint16_t* hid = A.hidden + (size_t)(A.layer0 + layer) * A.hidden_ls;
+  const uint16_t* wg = A.wg + (size_t)(A.layer0 + layer) * A.wg_ls;
+
+  const uint16_t* arow[MT][2];
+#pragma unroll
+  for (int m = 0; m < MT; ++m) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      long long r = tok0 + m * 16 + h * 8 + g;
+      if (r > T - 1) r = T - 1;  // rows past the end re-read the last row; results dropped
+      arow[m][h] = hid + r * A.ld_h + q * 8;
+    }
+  }
+  const uint16_t* brow[NT];
+  bool bval[NT];
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    const int e = n * 8 + g;
+    bval[n] = e < E;
+    brow[n] = wg + (long long)(bval[n] ? e : 0) * A.ld_w + q * 8;
+  }
+
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int m = 0; m < MT; ++m)
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[m][n][i] = 0.0f;
+
+  const int full_chunks = d / 32;
+  int kc = 0;
+  for (; kc + KU <= full_chunks; kc += KU) {
+    uint4 av[KU][MT][2];
+#pragma unroll
+    for (int u = 0; u < KU; ++u)
+#pragma unroll
+      for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) av[u][m][h] = ldg_stream(arow[m][h] + (kc + u) * 32);
+#pragma unroll
+    for (int u = 0; u < KU; ++u) {
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        uint4 b = make_uint4(0, 0, 0, 0);
+        if (bval[n]) b = __ldg(reinterpret_cast<const uint4*>(brow[n] + (kc + u) * 32));
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          mma_bf16_16816(acc[m][n], av[u][m][0].x, av[u][m][1].x, av[u][m][0].y, av[u][m][1].y,
+                         b.x, b.y);
+          mma_bf16_16816(acc[m][n], av[u][m][0].z, av[u][m][1].z, av[u][m][0].w, av[u][m][1].w,
+                         b.z, b.w);
+        }
+      }
+    }
+  }
+  // remaining chunks, the last possibly partial (d is a multiple of 8)
+  for (; kc * 32 < d; ++kc) {
+    const bool in = (kc * 32 + q * 8 + 8) <= d;
+    uint4 av[MT][2];
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+        av[m][h] = in ? ldg_stream(arow[m][h] + kc * 32) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      uint4 b = make_uint4(0, 0, 0, 0);
+      if (bval[n] && in) b = __ldg(reinterpret_cast<const uint4*>(brow[n] + kc * 32));
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        mma_bf16_16816(acc[m][n], av[m][0].x, av[m][1].x, av[m][0].y, av[m][1].y, b.x, b.y);
+        mma_bf16_16816(acc[m][n], av[m][0].z, av[m][1].z, av[m][0].w, av[m][1].w, b.z, b.w);
+      }
+    }
+  }
+
+  // accumulators (+ bias) -> this warp's shared-memory tile [ROWS][LDS]
+  float* tile = smem_tile + (size_t)warp * ROWS * LDS;
+  const float* bias = A.bias ? A.bias + (size_t)(A.layer0 + layer) * E : nullptr;
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    const int e0 = n * 8 + q * 2;
+    const float b0 = (bias && e0 < E) ? bias[e0] : 0.0f;
+    const float b1 = (bias && e0 + 1 < E) ? bias[e0 + 1] : 0.0f;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+      float v0 = acc[m][n][0], v1 = acc[m][n][1], v2 = acc[m][n][2], v3 = acc[m][n][3];
+      if (bias) {
+        v0 = __fadd_rn(v0, b0); v1 = __fadd_rn(v1, b1);
+        v2 = __fadd_rn(v2, b0); v3 = __fadd_rn(v3, b1);
+      }
+      const float big = 3.402823466e+38f;  // non-finite logits are clamped into range
+      v0 = fminf(fmaxf(v0, -big), big); v1 = fminf(fmaxf(v1, -big), big);
+      v2 = fminf(fmaxf(v2, -big), big); v3 = fminf(fmaxf(v3, -big), big);
+      tile[(m * 16 + g) * LDS + e0] = v0;
+      tile[(m * 16 + g) * LDS + e0 + 1] = v1;
+      tile[(m * 16 + g + 8) * LDS + e0] = v2;
+      tile[(m * 16 + g + 8) * LDS + e0 + 1] = v3;
+    }
+  }
+  __syncwarp();
+
+  const int rows_here = (int)min((long long)ROWS, (long long)T - tok0);
+  if (A.logits_out) {
+    float* out = A.logits_out + ((size_t)(A.layer0 + layer) * T + tok0) * E;
+    for (int idx = lane; idx < rows_here * E; idx += 32) {
+      const int r = idx / E, e = idx - r * E;
+      out[idx] = tile[r * LDS + e];
+    }
+  }
+
+  unsigned char* ws = A.ws + (size_t)(A.layer0 + layer) * A.ws_ls;
+  const int k = A.k, c = A.c;
+  for (int r = lane; r < rows_here; r += 32) {
+    const long long t = tok0 + r;
+    const size_t lt = (size_t)(A.layer0 + layer) * T + t;
+    token_epilogue(tile + r * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
+                   reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
+                   ws + A.lay.cand_ids + (size_t)t * c,
+                   reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
+                   A.expert_ids + lt * k, A.weights + lt * k);
+  }
+}
+
+}  // namespace laser

@@ -1,0 +1,295 @@
+// Host side of the C ABI declared in include/laser.h: validation, workspace carve-up,
+// kernel selection by E, launches.  No allocation, no synchronisation (except the host-
+// buffer entry point), no state between calls.
+#include "../../include/laser.h"
+
+#include "k1_router.cuh"
+#include "k2_select.cuh"
+#include "k3_dispatch.cuh"
+
+using namespace laser;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate_params(const laser_params* p) {
+  if (!p) return LASER_ERR_INVALID_ARG;
+  if (p->T < 0 || p->d <= 0 || p->E < 1 || p->E > LASER_MAX_EXPERTS) return LASER_ERR_INVALID_ARG;
+  if (p->k < 1 || p->k > p->c || p->c > p->E) return LASER_ERR_INVALID_ARG;
+  if (p->d % 8 != 0) return LASER_ERR_INVALID_ARG;
+  if (!(p->eps_high >= 0.0f) || !(p->t_fix >= 0.0f) || !(p->t_fix <= 1.0f))
+    return LASER_ERR_INVALID_ARG;
+  if (p->trim_mode == 1) return LASER_ERR_UNSUPPORTED;
+  if (p->trim_mode != 0) return LASER_ERR_INVALID_ARG;
+  if (p->update_granularity != 1) return LASER_ERR_UNSUPPORTED;
+  if (p->n_bins < 1) return LASER_ERR_INVALID_ARG;
+  if (p->ld_hidden < p->d || p->ld_w < p->d) return LASER_ERR_INVALID_ARG;
+  if (p->ld_hidden % 8 != 0 || p->ld_w % 8 != 0) return LASER_ERR_MISALIGNED;
+  if ((long long)p->T * p->k > 0x7fffffffLL) return LASER_ERR_INVALID_ARG;
+  return LASER_OK;
+}
+
+template <int NT, int MT, int KU>
+cudaError_t launch_k1(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  constexpr int rows_per_block = 4 * MT * 16;
+  const size_t smem = sizeof(float) * 4 * MT * 16 * (NT * 8 + 1);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k1_router_mma<NT, MT, KU>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((unsigned)((a.T + rows_per_block - 1) / rows_per_block), (unsigned)n_layers);
+  k1_router_mma<NT, MT, KU><<<grid, 128, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_k1_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  const int E = a.E;
+  if (E <= 8) return launch_k1<1, 2, 4>(a, n_layers, s);
+  if (E <= 16) return launch_k1<2, 2, 4>(a, n_layers, s);
+  if (E <= 32) return launch_k1<4, 2, 2>(a, n_layers, s);
+  if (E <= 64) return launch_k1<8, 2, 2>(a, n_layers, s);
+  if (E <= 128) return launch_k1<16, 1, 2>(a, n_layers, s);
+  return launch_k1<32, 1, 1>(a, n_layers, s);
+}
+
+int k2_tile_tokens(int c) { return c <= 128 ? 128 : 64; }
+
+size_t k2_smem_bytes(int E, int c) {
+  const int tile = k2_tile_tokens(c);
+  size_t off = align256(sizeof(int32_t) * E);
+  off = align256(off + sizeof(unsigned long long) * c);
+  const size_t buf = align256((size_t)tile * c) + align256(sizeof(uint16_t) * tile);
+  return off + 2 * buf;
+}
+
+// Enqueues all stages for layers [layer0, layer0 + n) of a batched call.
+int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const float* eps,
+                  const float* tfix, cudaStream_t s, void* const* ev) {
+  auto mark = [&](int i) {
+    return !ev || !ev[i] || cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), s) == cudaSuccess;
+  };
+  a.layer0 = layer0;
+  for (int l = 0; l < n; ++l) {
+    a.eps_high[l] = eps ? eps[layer0 + l] : p->eps_high;
+    a.t_fix[l] = tfix ? tfix[layer0 + l] : p->t_fix;
+  }
+  cudaError_t e = cudaSuccess;
+  if (!mark(0)) return LASER_ERR_CUDA;
+  if (a.T > 0) {
+    e = launch_k1_for_E(a, n, s);
+    if (e != cudaSuccess) return LASER_ERR_CUDA;
+    if (!mark(1)) return LASER_ERR_CUDA;
+    const size_t smem2 = k2_smem_bytes(a.E, a.c);
+    if (smem2 > 48 * 1024) {
+      e = cudaFuncSetAttribute(k2_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+      if (e != cudaSuccess) return LASER_ERR_CUDA;
+    }
+    k2_select<<<n, kK2Threads, smem2, s>>>(a, k2_tile_tokens(a.c));
+    if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+    dim3 gw((unsigned)((a.T + 255) / 256), (unsigned)n);
+    k2_weights<<<gw, 256, 0, s>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+  } else if (!mark(1)) {
+    return LASER_ERR_CUDA;
+  }
+  if (!mark(2)) return LASER_ERR_CUDA;
+  const size_t smem3 = sizeof(int32_t) * kK3Warps * a.E;
+  dim3 g3((unsigned)a.lay.n_blk, (unsigned)n);
+  k3_hist<<<g3, kK3Threads, smem3, s>>>(a);
+  if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+  k3_scan<<<n, kK3Threads, 0, s>>>(a);
+  if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+  k3_scatter<<<g3, kK3Threads, smem3, s>>>(a);
+  if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+  if (!mark(3)) return LASER_ERR_CUDA;
+  return LASER_OK;
+}
+
+}  // namespace
+
+extern "C" int laser_version(void) { return 100; }
+
+extern "C" const char* laser_strerror(int status) {
+  switch (status) {
+    case LASER_OK: return "ok";
+    case LASER_ERR_INVALID_ARG: return "invalid argument";
+    case LASER_ERR_UNSUPPORTED: return "unsupported mode";
+    case LASER_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LASER_ERR_MISALIGNED: return "pointer or row stride not 16-byte aligned";
+    case LASER_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int laser_workspace_bytes(const laser_params* p, size_t* bytes) {
+  if (!bytes) return LASER_ERR_INVALID_ARG;
+  const int rc = validate_params(p);
+  if (rc != LASER_OK) return rc;
+  *bytes = make_layout(p->T, p->E, p->k, p->c).total;
+  return LASER_OK;
+}
+
+extern "C" int laser_route_layers_profiled(
+    int32_t n_layers, const void* hidden, const void* w_g, const float* bias, int32_t* loads,
+    const int32_t* expert_to_bin, int32_t* bin_loads, const laser_params* p,
+    const float* eps_high_per_layer, const float* t_fix_per_layer, int32_t* expert_ids,
+    float* weights, int32_t* offsets, int32_t* perm, float* logits_out, int32_t* status_word,
+    void* workspace, size_t workspace_bytes, void* cuda_stream, void* const* stage_events) {
+  const int rc = validate_params(p);
+  if (rc != LASER_OK) return rc;
+  if (n_layers < 1) return LASER_ERR_INVALID_ARG;
+  if (!w_g || !loads || !offsets || !workspace) return LASER_ERR_INVALID_ARG;
+  if (p->T > 0 && (!hidden || !expert_ids || !weights || !perm)) return LASER_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_g)) return LASER_ERR_MISALIGNED;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LASER_ERR_MISALIGNED;
+  for (int l = 0; l < n_layers; ++l) {
+    const float e = eps_high_per_layer ? eps_high_per_layer[l] : p->eps_high;
+    const float t = t_fix_per_layer ? t_fix_per_layer[l] : p->t_fix;
+    if (!(e >= 0.0f) || !(t >= 0.0f) || !(t <= 1.0f)) return LASER_ERR_INVALID_ARG;
+  }
+  const WorkspaceLayout lay = make_layout(p->T, p->E, p->k, p->c);
+  if (workspace_bytes < lay.total * (size_t)n_layers) return LASER_ERR_WORKSPACE_TOO_SMALL;
+
+  RouteArgs a;
+  a.hidden = static_cast<const uint16_t*>(hidden);
+  a.hidden_ls = (long long)p->T * p->ld_hidden;
+  a.wg = static_cast<const uint16_t*>(w_g);
+  a.wg_ls = (long long)p->E * p->ld_w;
+  a.bias = bias;
+  a.loads = loads;
+  a.e2b = expert_to_bin;
+  a.bin_loads = bin_loads;
+  a.expert_ids = expert_ids;
+  a.weights = weights;
+  a.offsets = offsets;
+  a.perm = perm;
+  a.logits_out = logits_out;
+  a.status = status_word;
+  a.ws = static_cast<unsigned char*>(workspace);
+  a.ws_ls = lay.total;
+  a.lay = lay;
+  a.T = p->T; a.d = p->d; a.E = p->E; a.k = p->k; a.c = p->c;
+  a.n_bins = p->n_bins; a.renorm = p->renormalize ? 1 : 0;
+  a.ld_h = p->ld_hidden; a.ld_w = p->ld_w;
+
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  for (int l0 = 0; l0 < n_layers; l0 += kMaxLayersPerLaunch) {
+    const int n = n_layers - l0 < kMaxLayersPerLaunch ? n_layers - l0 : kMaxLayersPerLaunch;
+    const int r = enqueue_group(a, l0, n, p, eps_high_per_layer, t_fix_per_layer, s, stage_events);
+    if (r != LASER_OK) return r;
+  }
+  return LASER_OK;
+}
+
+extern "C" int laser_route_layers(int32_t n_layers, const void* hidden, const void* w_g,
+                                  const float* bias, int32_t* loads,
+                                  const int32_t* expert_to_bin, int32_t* bin_loads,
+                                  const laser_params* p, const float* eps_high_per_layer,
+                                  const float* t_fix_per_layer, int32_t* expert_ids,
+                                  float* weights, int32_t* offsets, int32_t* perm,
+                                  float* logits_out, int32_t* status_word, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+  return laser_route_layers_profiled(n_layers, hidden, w_g, bias, loads, expert_to_bin, bin_loads,
+                                     p, eps_high_per_layer, t_fix_per_layer, expert_ids, weights,
+                                     offsets, perm, logits_out, status_word, workspace,
+                                     workspace_bytes, cuda_stream, nullptr);
+}
+
+extern "C" int laser_route(const void* hidden, const void* w_g, const float* bias, int32_t* loads,
+                           const int32_t* expert_to_bin, int32_t* bin_loads,
+                           const laser_params* p, int32_t* expert_ids, float* weights,
+                           int32_t* offsets, int32_t* perm, float* logits_out,
+                           int32_t* status_word, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream) {
+  return laser_route_layers(1, hidden, w_g, bias, loads, expert_to_bin, bin_loads, p, nullptr,
+                            nullptr, expert_ids, weights, offsets, perm, logits_out, status_word,
+                            workspace, workspace_bytes, cuda_stream);
+}
+
+namespace {
+struct HostArena {
+  size_t hidden, wg, bias, loads, e2b, bins, ids, weights, offsets, perm, status, ws, total;
+};
+HostArena make_arena(int L, const laser_params* p) {
+  HostArena h;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
+  h.hidden = take(2ull * L * p->T * p->ld_hidden);
+  h.wg = take(2ull * L * p->E * p->ld_w);
+  h.bias = take(4ull * L * p->E);
+  h.loads = take(4ull * L * p->E);
+  h.e2b = take(4ull * p->E);
+  h.bins = take(4ull * L * p->n_bins);
+  h.ids = take(4ull * L * p->T * p->k);
+  h.weights = take(4ull * L * p->T * p->k);
+  h.offsets = take(4ull * L * (p->E + 1));
+  h.perm = take(4ull * L * p->T * p->k);
+  h.status = take(4);
+  h.ws = take(make_layout(p->T, p->E, p->k, p->c).total * (size_t)L);
+  h.total = off;
+  return h;
+}
+}  // namespace
+
+extern "C" int laser_host_arena_bytes(int32_t n_layers, const laser_params* p, size_t* bytes) {
+  if (!bytes || n_layers < 1) return LASER_ERR_INVALID_ARG;
+  const int rc = validate_params(p);
+  if (rc != LASER_OK) return rc;
+  *bytes = make_arena(n_layers, p).total;
+  return LASER_OK;
+}
+
+extern "C" int laser_route_host(int32_t n_layers, const void* hidden, const void* w_g,
+                                const float* bias, int32_t* loads, const int32_t* expert_to_bin,
+                                int32_t* bin_loads, const laser_params* p,
+                                const float* eps_high_per_layer, const float* t_fix_per_layer,
+                                int32_t* expert_ids, float* weights, int32_t* offsets,
+                                int32_t* perm, int32_t* status_out, void* arena,
+                                size_t arena_bytes, void* cuda_stream) {
+  const int rc = validate_params(p);
+  if (rc != LASER_OK) return rc;
+  if (n_layers < 1 || !arena || !w_g || !loads || !offsets) return LASER_ERR_INVALID_ARG;
+  if (p->T > 0 && (!hidden || !expert_ids || !weights || !perm)) return LASER_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return LASER_ERR_MISALIGNED;
+  const HostArena h = make_arena(n_layers, p);
+  if (arena_bytes < h.total) return LASER_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* base = static_cast<unsigned char*>(arena);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t L = (size_t)n_layers, T = (size_t)p->T, E = (size_t)p->E, k = (size_t)p->k;
+#define LASER_COPY(dst, src, bytes, kind)                                             \
+  do {                                                                                \
+    if ((bytes) > 0 && cudaMemcpyAsync((dst), (src), (bytes), (kind), s) != cudaSuccess) \
+      return LASER_ERR_CUDA;                                                          \
+  } while (0)
+  LASER_COPY(base + h.hidden, hidden, 2 * L * T * p->ld_hidden, cudaMemcpyHostToDevice);
+  LASER_COPY(base + h.wg, w_g, 2 * L * E * p->ld_w, cudaMemcpyHostToDevice);
+  if (bias) LASER_COPY(base + h.bias, bias, 4 * L * E, cudaMemcpyHostToDevice);
+  LASER_COPY(base + h.loads, loads, 4 * L * E, cudaMemcpyHostToDevice);
+  if (expert_to_bin) LASER_COPY(base + h.e2b, expert_to_bin, 4 * E, cudaMemcpyHostToDevice);
+  if (bin_loads) LASER_COPY(base + h.bins, bin_loads, 4 * L * p->n_bins, cudaMemcpyHostToDevice);
+  if (cudaMemsetAsync(base + h.status, 0, 4, s) != cudaSuccess) return LASER_ERR_CUDA;
+
+  const int r = laser_route_layers(
+      n_layers, base + h.hidden, base + h.wg, bias ? reinterpret_cast<float*>(base + h.bias) : nullptr,
+      reinterpret_cast<int32_t*>(base + h.loads),
+      expert_to_bin ? reinterpret_cast<int32_t*>(base + h.e2b) : nullptr,
+      bin_loads ? reinterpret_cast<int32_t*>(base + h.bins) : nullptr, p, eps_high_per_layer,
+      t_fix_per_layer, reinterpret_cast<int32_t*>(base + h.ids),
+      reinterpret_cast<float*>(base + h.weights), reinterpret_cast<int32_t*>(base + h.offsets),
+      reinterpret_cast<int32_t*>(base + h.perm), nullptr,
+      reinterpret_cast<int32_t*>(base + h.status), base + h.ws, h.total - h.ws, s);
+  if (r != LASER_OK) return r;
+
+  LASER_COPY(expert_ids, base + h.ids, 4 * L * T * k, cudaMemcpyDeviceToHost);
+  LASER_COPY(weights, base + h.weights, 4 * L * T * k, cudaMemcpyDeviceToHost);
+  LASER_COPY(offsets, base + h.offsets, 4 * L * (E + 1), cudaMemcpyDeviceToHost);
+  LASER_COPY(perm, base + h.perm, 4 * L * T * k, cudaMemcpyDeviceToHost);
+  LASER_COPY(loads, base + h.loads, 4 * L * E, cudaMemcpyDeviceToHost);
+  if (bin_loads) LASER_COPY(bin_loads, base + h.bins, 4 * L * p->n_bins, cudaMemcpyDeviceToHost);
+  if (status_out) LASER_COPY(status_out, base + h.status, 4, cudaMemcpyDeviceToHost);
+#undef LASER_COPY
+  if (cudaStreamSynchronize(s) != cudaSuccess) return LASER_ERR_CUDA;
+  return LASER_OK;
+}

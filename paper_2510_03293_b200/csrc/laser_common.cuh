@@ -1,0 +1,84 @@
+// Shared device helpers and the per-layer argument block of the LASER routing kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace laser {
+
+constexpr int kMaxLayersPerLaunch = 64;
+constexpr int kMaxExperts = 256;
+
+// Scratch carved from the caller's workspace for one layer.  Offsets in bytes.
+struct WorkspaceLayout {
+  size_t cstar;        // uint16 [T]        0 = top-k branch, else c*
+  size_t cand_ids;     // uint8  [T, c]     ranking pi(0..c-1)
+  size_t cand_scores;  // float  [T, c]     s_pi(j)
+  size_t sel_rank;     // uint8  [T, k]     rank positions chosen by the load-aware scan
+  size_t blk_hist;     // int32  [n_blk, E] dispatch block histograms, then block bases
+  size_t total;        // bytes per layer, multiple of 256
+  int n_blk;           // dispatch blocks per layer
+};
+
+constexpr int kDispatchPairsPerBlock = 4096;
+
+__host__ __device__ inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+inline WorkspaceLayout make_layout(int T, int E, int k, int c) {
+  WorkspaceLayout w;
+  size_t off = 0;
+  w.cstar = off;        off = align256(off + sizeof(uint16_t) * (size_t)T);
+  w.cand_ids = off;     off = align256(off + (size_t)T * c);
+  w.cand_scores = off;  off = align256(off + sizeof(float) * (size_t)T * c);
+  w.sel_rank = off;     off = align256(off + (size_t)T * k);
+  long long pairs = (long long)T * k;
+  w.n_blk = (int)((pairs + kDispatchPairsPerBlock - 1) / kDispatchPairsPerBlock);
+  if (w.n_blk < 1) w.n_blk = 1;
+  w.blk_hist = off;     off = align256(off + sizeof(int32_t) * (size_t)w.n_blk * E);
+  w.total = off;
+  return w;
+}
+
+// Kernel-side view of one batched call: layer l uses base + l * stride of every array.
+struct RouteArgs {
+  const uint16_t* hidden;  long long hidden_ls;   // elements
+  const uint16_t* wg;      long long wg_ls;
+  const float* bias;       // [L, E] or null
+  int32_t* loads;          // [L, E]
+  const int32_t* e2b;      // [E] or null
+  int32_t* bin_loads;      // [L, B] or null
+  int32_t* expert_ids;     // [L, T, k]
+  float* weights;          // [L, T, k]
+  int32_t* offsets;        // [L, E+1]
+  int32_t* perm;           // [L, T*k]
+  float* logits_out;       // [L, T, E] or null
+  int32_t* status;         // device status word or null
+  unsigned char* ws;       size_t ws_ls;          // bytes
+  WorkspaceLayout lay;
+  int T, d, E, k, c, n_bins, renorm;
+  long long ld_h, ld_w;
+  int layer0;              // first layer of this launch
+  float eps_high[kMaxLayersPerLaunch];
+  float t_fix[kMaxLayersPerLaunch];
+};
+
+// fp32 exponential for y <= 0 with a fixed sequence of correctly rounded operations:
+//   y < -80 -> 0;  n = rint(y*log2e);  r = y - n*ln2 (two fma steps);
+//   degree-7 Taylor polynomial in Horner form;  result = p * 2^n.
+__device__ __forceinline__ float exp32(float y) {
+  if (y < -80.0f) return 0.0f;
+  float n = rintf(__fmul_rn(y, __uint_as_float(0x3FB8AA3Bu)));
+  float r = __fmaf_rn(n, -__uint_as_float(0x3F317200u), y);
+  r = __fmaf_rn(n, -__uint_as_float(0x35BFBE8Eu), r);
+  float p = __uint_as_float(0x39500D01u);
+  p = __fmaf_rn(p, r, __uint_as_float(0x3AB60B61u));
+  p = __fmaf_rn(p, r, __uint_as_float(0x3C088889u));
+  p = __fmaf_rn(p, r, __uint_as_float(0x3D2AAAABu));
+  p = __fmaf_rn(p, r, __uint_as_float(0x3E2AAAABu));
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  int ni = __float2int_rn(n);                       // in [-116, 0]
+  return __fmul_rn(p, __int_as_float((ni + 127) << 23));
+}
+
+}  // namespace laser

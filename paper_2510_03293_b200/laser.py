@@ -1,0 +1,217 @@
+"""Python binding of the LASER routing C ABI (``include/laser.h``).
+
+Argument marshalling only: every step of the routing path runs in the CUDA kernels of
+``liblaser.so``.  torch is used for device memory and streams.  There is no fallback: if the
+shared library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblaser.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build the CUDA library first "
+        "(python -c 'import __graft_entry__ as g; g.build()'); there is no CPU fallback")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED = -2
+ERR_WORKSPACE_TOO_SMALL = -3
+ERR_MISALIGNED = -4
+ERR_CUDA = -5
+DEV_LOAD_OVERFLOW = 1
+MAX_EXPERTS = 256
+
+EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_route",
+           "laser_route_layers", "laser_route_layers_profiled", "laser_host_arena_bytes",
+           "laser_route_host")
+
+
+class LaserParams(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int32), ("d", ctypes.c_int32), ("E", ctypes.c_int32),
+                ("k", ctypes.c_int32), ("c", ctypes.c_int32),
+                ("eps_high", ctypes.c_float), ("t_fix", ctypes.c_float),
+                ("trim_mode", ctypes.c_int32), ("update_granularity", ctypes.c_int32),
+                ("renormalize", ctypes.c_int32), ("n_bins", ctypes.c_int32),
+                ("ld_hidden", ctypes.c_int64), ("ld_w", ctypes.c_int64),
+                ("seed", ctypes.c_uint64)]
+
+
+_vp, _i32, _sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+_pp = ctypes.POINTER(LaserParams)
+_lib.laser_version.restype = ctypes.c_int
+_lib.laser_strerror.argtypes = [ctypes.c_int]
+_lib.laser_strerror.restype = ctypes.c_char_p
+_lib.laser_workspace_bytes.argtypes = [_pp, ctypes.POINTER(_sz)]
+_lib.laser_workspace_bytes.restype = ctypes.c_int
+_lib.laser_route.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _pp, _vp, _vp, _vp, _vp, _vp, _vp,
+                             _vp, _sz, _vp]
+_lib.laser_route.restype = ctypes.c_int
+_lib.laser_route_layers.argtypes = [_i32, _vp, _vp, _vp, _vp, _vp, _vp, _pp, _vp, _vp,
+                                    _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.laser_route_layers.restype = ctypes.c_int
+_lib.laser_route_layers_profiled.argtypes = _lib.laser_route_layers.argtypes + [_vp]
+_lib.laser_route_layers_profiled.restype = ctypes.c_int
+_lib.laser_host_arena_bytes.argtypes = [_i32, _pp, ctypes.POINTER(_sz)]
+_lib.laser_host_arena_bytes.restype = ctypes.c_int
+_lib.laser_route_host.argtypes = [_i32, _vp, _vp, _vp, _vp, _vp, _vp, _pp, _vp, _vp,
+                                  _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.laser_route_host.restype = ctypes.c_int
+
+
+class LaserError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"laser: {strerror(status)} ({status})")
+
+
+def version() -> int:
+    return int(_lib.laser_version())
+
+
+def strerror(status: int) -> str:
+    return _lib.laser_strerror(int(status)).decode()
+
+
+def make_params(T, d, E, k, c, eps_high, t_fix, renormalize=1, n_bins=1, ld_hidden=None,
+                ld_w=None, trim_mode=0, update_granularity=1, seed=0) -> LaserParams:
+    return LaserParams(T, d, E, k, c, eps_high, t_fix, trim_mode, update_granularity,
+                       int(renormalize), n_bins, d if ld_hidden is None else ld_hidden,
+                       d if ld_w is None else ld_w, seed)
+
+
+def workspace_bytes(p: LaserParams) -> int:
+    out = _sz(0)
+    rc = _lib.laser_workspace_bytes(ctypes.byref(p), ctypes.byref(out))
+    if rc != OK:
+        raise LaserError(rc)
+    return int(out.value)
+
+
+def host_arena_bytes(n_layers: int, p: LaserParams) -> int:
+    out = _sz(0)
+    rc = _lib.laser_host_arena_bytes(n_layers, ctypes.byref(p), ctypes.byref(out))
+    if rc != OK:
+        raise LaserError(rc)
+    return int(out.value)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _floats(v: Optional[Sequence[float]]):
+    if v is None:
+        return None, None
+    arr = (ctypes.c_float * len(v))(*[float(x) for x in v])
+    return arr, ctypes.cast(arr, _vp)
+
+
+def route_raw(hidden, w_g, bias, loads, expert_to_bin, bin_loads, p, expert_ids, weights,
+              offsets, perm, logits_out, status_word, workspace, workspace_nbytes,
+              stream=0) -> int:
+    """laser_route with raw integer device addresses (or None); returns the status code."""
+    return int(_lib.laser_route(hidden, w_g, bias, loads, expert_to_bin, bin_loads,
+                                ctypes.byref(p), expert_ids, weights, offsets, perm, logits_out,
+                                status_word, workspace, workspace_nbytes, stream))
+
+
+@dataclass
+class RouteResult:
+    expert_ids: "object"
+    weights: "object"
+    offsets: "object"
+    perm: "object"
+    loads: "object"
+    bin_loads: "object"
+    logits: "object"
+    status: "object"
+
+
+def route_layers(hidden, w_g, bias, loads, p: LaserParams, *, expert_to_bin=None,
+                 bin_loads=None, eps_high=None, t_fix=None, want_logits=False, out=None,
+                 workspace=None, stream=None, stage_events=None) -> RouteResult:
+    """laser_route_layers on torch CUDA tensors.
+
+    hidden [L,T,d] bf16, w_g [L,E,d] bf16, bias [L,E] f32 or None, loads [L,E] int32
+    (updated in place), bin_loads [L,B] int32 or None (updated in place).  ``out`` may carry
+    preallocated outputs from an earlier RouteResult; otherwise they are allocated here.
+    ``stage_events``: four torch.cuda.Event objects (already recorded once, so that their
+    handles exist) to be recorded between the stages.
+    """
+    import torch
+
+    L = hidden.shape[0]
+    dev = hidden.device
+    T, E, k = p.T, p.E, p.k
+    if out is None:
+        out = RouteResult(
+            torch.empty((L, T, k), dtype=torch.int32, device=dev),
+            torch.empty((L, T, k), dtype=torch.float32, device=dev),
+            torch.empty((L, E + 1), dtype=torch.int32, device=dev),
+            torch.empty((L, T * k), dtype=torch.int32, device=dev),
+            loads, bin_loads,
+            torch.empty((L, T, E), dtype=torch.float32, device=dev) if want_logits else None,
+            torch.zeros((1,), dtype=torch.int32, device=dev))
+    need = workspace_bytes(p) * L
+    if workspace is None:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+    eps_arr, eps_p = _floats(eps_high)
+    tf_arr, tf_p = _floats(t_fix)
+    s = torch.cuda.current_stream(dev) if stream is None else stream
+    ev_p = None
+    if stage_events is not None:
+        ev_arr = (_vp * 4)(*[int(e.cuda_event) for e in stage_events])
+        ev_p = ctypes.cast(ev_arr, _vp)
+    rc = _lib.laser_route_layers_profiled(
+        L, _ptr(hidden), _ptr(w_g), _ptr(bias), _ptr(loads), _ptr(expert_to_bin),
+        _ptr(bin_loads), ctypes.byref(p), eps_p, tf_p, _ptr(out.expert_ids), _ptr(out.weights),
+        _ptr(out.offsets), _ptr(out.perm), _ptr(out.logits), _ptr(out.status),
+        _ptr(workspace), workspace.numel(), s.cuda_stream, ev_p)
+    if rc != OK:
+        raise LaserError(rc)
+    return out
+
+
+def route(hidden, w_g, bias, loads, p: LaserParams, *, bin_loads=None, **kw) -> RouteResult:
+    """laser_route for one layer: hidden [T,d], w_g [E,d], bias [E], loads [E] (in place)."""
+    r = route_layers(hidden[None], w_g[None], None if bias is None else bias[None], loads[None],
+                     p, bin_loads=None if bin_loads is None else bin_loads[None], **kw)
+    return RouteResult(r.expert_ids[0], r.weights[0], r.offsets[0], r.perm[0], loads, bin_loads,
+                       None if r.logits is None else r.logits[0], r.status)
+
+
+def route_host(hidden, w_g, bias, loads, p: LaserParams, arena, *, expert_to_bin=None,
+               bin_loads=None, eps_high=None, t_fix=None, out=None, stream=None):
+    """laser_route_host: every array is a HOST (ideally pinned) torch tensor except ``arena``
+    (device uint8 tensor of at least host_arena_bytes).  Returns (expert_ids, weights,
+    offsets, perm, status) host tensors; loads / bin_loads are updated in place."""
+    import torch
+
+    L = hidden.shape[0]
+    T, E, k = p.T, p.E, p.k
+    if out is None:
+        pin = dict(pin_memory=True)
+        out = (torch.empty((L, T, k), dtype=torch.int32, **pin),
+               torch.empty((L, T, k), dtype=torch.float32, **pin),
+               torch.empty((L, E + 1), dtype=torch.int32, **pin),
+               torch.empty((L, T * k), dtype=torch.int32, **pin),
+               torch.zeros((1,), dtype=torch.int32, **pin))
+    eps_arr, eps_p = _floats(eps_high)
+    tf_arr, tf_p = _floats(t_fix)
+    s = torch.cuda.current_stream(arena.device) if stream is None else stream
+    rc = _lib.laser_route_host(
+        L, _ptr(hidden), _ptr(w_g), _ptr(bias), _ptr(loads), _ptr(expert_to_bin),
+        _ptr(bin_loads), ctypes.byref(p), eps_p, tf_p, _ptr(out[0]), _ptr(out[1]), _ptr(out[2]),
+        _ptr(out[3]), _ptr(out[4]), _ptr(arena), arena.numel(), s.cuda_stream)
+    if rc != OK:
+        raise LaserError(rc)
+    return out
