@@ -51,6 +51,18 @@ def workload_config(w, n_layers):
                      (2.0 * n_layers * w.T * w.d / 1e9)}
 
 
+def launches_per_step(w, L) -> int:
+    """Kernels the library enqueues per step: router + selection per token chunk, then the
+    four dispatch kernels, per group of at most 64 layers."""
+    chunk = int(os.environ.get("LASER_CHUNK_TOKENS", "4096") or 4096)
+    chunk = -(-chunk // 256) * 256
+    n_chunks = -(-w.T // chunk)
+    while n_chunks > 16:
+        chunk *= 2
+        n_chunks = -(-w.T // chunk)
+    return (2 * n_chunks + 4) * ((L + 63) // 64)
+
+
 # --------------------------------------------------------------------------- CPU oracle arm
 def oracle_pass(oracle, np, layers_data, w, eps, tfix):
     """The oracle's whole path on a list of (hidden_bits, wg_bits, bias) layers."""
@@ -242,7 +254,7 @@ def run_gpu(args, w):
         "path": {"k1_ms": k1, "k2_ms": k2, "k3_ms": k3, "path_gbs": path_gbs,
                  "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
         "routing": {"mean_imbalance_max_over_mean": imb, "status_word": status},
-        "gpu_launches": 6 * ((L + 63) // 64) * args.steps,
+        "gpu_launches": launches_per_step(w, L) * args.steps,
         "clocks": clocks,
     }
 

@@ -16,10 +16,15 @@
  *
  * General rules for every entry point
  *   - Pointers are DEVICE pointers unless the parameter is documented as host.
- *   - The caller owns every buffer; the library keeps no state between calls.
+ *   - The caller owns every buffer; no routing state is kept between calls.
  *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*); the call
  *     returns without synchronising, except laser_route_host, which synchronises the stream
- *     before returning.
+ *     before returning.  Calls with more tokens than one chunk (4096 by default, environment
+ *     variable LASER_CHUNK_TOKENS) overlap the ordered selection of one chunk with the router
+ *     kernel of the next on a library-owned high-priority side stream; that stream and a few
+ *     events are created per device on the first such call and live until the process
+ *     exits.  The side work is joined back into the caller's stream before the call's last
+ *     kernels, so stream order as seen by the caller is unchanged.
  *   - Return value: LASER_OK (0) or a negative status.  On a validation error nothing is
  *     launched and no output is touched.
  *   - Conditions only visible on the device are OR-ed into *status_word (device int32,
@@ -44,7 +49,9 @@ enum {
   LASER_ERR_CUDA = -5              /* a CUDA runtime call failed (launch error) */
 };
 
-enum { LASER_DEV_LOAD_OVERFLOW = 1 }; /* bit in *status_word: a load counter passed 2^31-1 */
+/* Bit in *status_word: on entry some load counter was negative or within T of 2^31-1, so it
+ * could overflow during the call; the call's results are then unspecified. */
+enum { LASER_DEV_LOAD_OVERFLOW = 1 };
 
 enum { LASER_MAX_EXPERTS = 256 };
 
@@ -103,7 +110,7 @@ int laser_workspace_bytes(const laser_params* p, size_t* bytes);
  *   bin_loads   [n_bins] int32 in/out, or NULL to skip bin accounting
  *   p           host
  *   expert_ids  [T, k] int32 out.  Top-k branch: descending score.  Expanded branch:
- *               ascending (load, score rank).
+ *               ascending (load seen by the token, score rank).
  *   weights     [T, k] fp32 out, weights[t,j] belongs to expert_ids[t,j]
  *   offsets     [E+1] int32 out, exclusive prefix of this call's per-expert counts
  *   perm        [T*k] int32 out: pair ids t*k+j grouped by expert, ascending within an expert

@@ -98,8 +98,8 @@ __global__ void __launch_bounds__(128) k1_router_mma(const RouteArgs A) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, q = lane & 3;
   const int T = A.T, d = A.d, E = A.E;
-  const long long tok0 = ((long long)blockIdx.x * 4 + warp) * ROWS;
-  if (tok0 >= T) return;
+  const long long tok0 = A.tok_begin + ((long long)blockIdx.x * 4 + warp) * ROWS;
+  if (tok0 >= A.tok_end) return;
 
   const uint16_t* hid = A.hidden + (size_t)(A.layer0 + layer) * A.hidden_ls;
   const uint16_t* wg = A.wg + (size_t)(A.layer0 + layer) * A.wg_ls;
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(128) k1_router_mma(const RouteArgs A) {
   }
   __syncwarp();
 
-  const int rows_here = (int)min((long long)ROWS, (long long)T - tok0);
+  const int rows_here = (int)min((long long)ROWS, (long long)A.tok_end - tok0);
   if (A.logits_out) {
     float* out = A.logits_out + ((size_t)(A.layer0 + layer) * T + tok0) * E;
     for (int idx = lane; idx < rows_here * E; idx += 32) {

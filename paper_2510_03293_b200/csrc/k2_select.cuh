@@ -1,145 +1,239 @@
 // K2: the ordered, load-aware selection (Algorithm 1, StableSortByLoad + first k) and the
-// per-token load update.  Tokens of one layer form one dependency chain, so one warp per
-// layer walks them in row order with the load vector in shared memory; the other warps of
-// the block only stage the next tile of candidate records.  Layers are independent blocks.
+// per-token load update.  Tokens of one layer form one dependency chain; layers are
+// independent thread blocks.
+//
+// Only tokens whose candidate set is larger than k (c* > k, "decision tokens") have a
+// load-dependent choice.  Every other token (top-k branch, or c* == k) sends its k best
+// experts whatever the loads are, so its increments are known without the chain.  The block
+// therefore splits the work:
+//   prep warps   stage a tile of candidate records in shared memory and, per group of 32
+//                tokens, count the fixed increments per expert (group totals) and, for every
+//                candidate of every decision token, the fixed increments of earlier tokens
+//                of the same group (ballot + popcount);
+//   chain warp   walks the decision tokens only: load seen by candidate j =
+//                L[e_j] (all earlier groups + earlier decisions) + its in-group prefix;
+//                ranks the candidates by (load, score rank) with warp shuffles, bumps the
+//                k winners, and adds the group totals at each group end.
+// The slot order of c* == k tokens, which depends on the loads they saw, is reconstructed
+// afterwards from the dispatch ranks (k3_finalize).
 #pragma once
 #include "laser_common.cuh"
 
 namespace laser {
 
-constexpr int kK2Threads = 128;
+constexpr int kK2Threads = 256;
+constexpr int kK2PrepWarps = kK2Threads / 32 - 1;
+constexpr int kK2Tile = 256;             // tokens per shared-memory buffer
+constexpr int kK2Groups = kK2Tile / 32;
+constexpr int kK2FastMaxLoad = 1 << 26;  // 32-bit keys (load << 5 | rank) need loads below this
 
-__device__ __forceinline__ void k2_stage_tile(uint8_t* dst_ids, uint16_t* dst_cs,
-                                              const uint8_t* src_ids, const uint16_t* src_cs,
-                                              int ntok, int c, int tid, int nthreads) {
-  const int bytes = ntok * c;
-  const int n16 = bytes >> 4;
-  const uint4* s4 = reinterpret_cast<const uint4*>(src_ids);
-  uint4* d4 = reinterpret_cast<uint4*>(dst_ids);
-  for (int i = tid; i < n16; i += nthreads) d4[i] = s4[i];
-  for (int i = (n16 << 4) + tid; i < bytes; i += nthreads) dst_ids[i] = src_ids[i];
-  for (int i = tid; i < ntok; i += nthreads) dst_cs[i] = src_cs[i];
+struct K2Buffers {
+  uint8_t* ids;     // [kK2Tile * c] ranked candidate ids
+  uint8_t* pre;     // [kK2Tile * c] in-group fixed increments seen by each candidate
+  uint16_t* cs;     // [kK2Tile]
+  int32_t* gtot;    // [kK2Groups * E] fixed increments per group and expert
+};
+
+__host__ __device__ inline size_t k2_buffer_bytes(int E, int c) {
+  return 2 * align256((size_t)kK2Tile * c) + align256(sizeof(uint16_t) * kK2Tile) +
+         align256(sizeof(int32_t) * kK2Groups * E);
 }
 
-// Adds one to a load counter; a counter at INT32_MAX stays there and raises the status bit.
-__device__ __forceinline__ void bump_load(int32_t* L, int e, int32_t* status) {
-  const int32_t v = L[e];
-  if (v == 0x7fffffff) { if (status) atomicOr(status, 1); }
-  else L[e] = v + 1;
+__device__ __forceinline__ K2Buffers k2_carve(unsigned char* base, int E, int c) {
+  K2Buffers b;
+  b.ids = base;
+  b.pre = base + align256((size_t)kK2Tile * c);
+  b.cs = reinterpret_cast<uint16_t*>(base + 2 * align256((size_t)kK2Tile * c));
+  b.gtot = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(b.cs) +
+                                      align256(sizeof(uint16_t) * kK2Tile));
+  return b;
 }
 
-// Dynamic shared memory: int32 L[E] | uint64 keys[c] | 2 x (uint8 ids[TILE*c], uint16 cs[TILE])
-__global__ void __launch_bounds__(kK2Threads) k2_select(const RouteArgs A, int tile_tokens) {
+// Prepares one group of 32 tokens (lane = token) of a tile.
+__device__ __forceinline__ void k2_prep_group(const K2Buffers& b, int g, int ntok,
+                                              const uint8_t* g_ids, const uint16_t* g_cs, int E,
+                                              int k, int c, int lane) {
+  const int tok = g * 32 + lane;
+  const bool valid = tok < ntok;
+  const int n_here = min(32, ntok - g * 32);
+  // stage this group's records
+  {
+    const int bytes = n_here * c;
+    const uint8_t* src = g_ids + (size_t)g * 32 * c;
+    uint8_t* dst = b.ids + (size_t)g * 32 * c;
+    const int n16 = bytes >> 4;
+    for (int i = lane; i < n16; i += 32)
+      reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+    for (int i = (n16 << 4) + lane; i < bytes; i += 32) dst[i] = src[i];
+  }
+  const int cs = valid ? g_cs[tok] : 0;
+  b.cs[tok] = (uint16_t)cs;
+  int32_t* gt = b.gtot + g * E;
+  for (int e = lane; e < E; e += 32) gt[e] = 0;
+  __syncwarp();
+  const bool fixed = valid && cs <= k;
+  const uint8_t* my = b.ids + (size_t)tok * c;
+  if (fixed)
+    for (int j = 0; j < k; ++j) atomicAdd(&gt[my[j]], 1);
+  unsigned dmask = __ballot_sync(0xffffffffu, valid && cs > k);
+  while (dmask) {
+    const int dl = __ffs(dmask) - 1;
+    dmask &= dmask - 1;
+    const int csd = __shfl_sync(0xffffffffu, cs, dl);
+    const uint8_t* cand = b.ids + (size_t)(g * 32 + dl) * c;
+    const unsigned before = (1u << dl) - 1;
+    int mine = 0;
+    for (int r = 0; r < csd; ++r) {
+      const int e = cand[r];
+      bool hit = false;
+      if (fixed)
+        for (int j = 0; j < k; ++j) hit |= (my[j] == e);
+      const int cnt = __popc(__ballot_sync(0xffffffffu, hit) & before);
+      if (lane == (r & 31)) mine = cnt;
+      if ((r & 31) == 31 || r == csd - 1) {
+        const int rr = (r & ~31) + lane;
+        if (rr <= r) b.pre[(size_t)(g * 32 + dl) * c + rr] = (uint8_t)mine;
+      }
+    }
+  }
+}
+
+// Chain over one tile, candidate sets no wider than a warp, loads below 2^26.
+template <int CMAX>
+__device__ __forceinline__ void k2_chain_tile(int32_t* L, const K2Buffers& b, int ntok, int E,
+                                              int k, int c, uint8_t* g_sel, int lane) {
+  const int n_groups = (ntok + 31) >> 5;
+  for (int g = 0; g < n_groups; ++g) {
+    const int tok = g * 32 + lane;
+    const int cs_l = tok < ntok ? b.cs[tok] : 0;
+    unsigned dmask = __ballot_sync(0xffffffffu, cs_l > k);
+    while (dmask) {
+      const int dl = __ffs(dmask) - 1;
+      dmask &= dmask - 1;
+      const int csd = __shfl_sync(0xffffffffu, cs_l, dl);
+      const size_t td = (size_t)(g * 32 + dl);
+      const bool mine = lane < csd;
+      const int id = mine ? b.ids[td * c + lane] : 0;
+      const int p = mine ? b.pre[td * c + lane] : 0;
+      const int32_t Lraw = mine ? L[id] : 0;
+      const uint32_t key = mine ? (((uint32_t)(Lraw + p) << 5) | (uint32_t)lane) : 0xffffffffu;
+      int cnt = 0;
+#pragma unroll
+      for (int j = 0; j < CMAX; ++j) {
+        const uint32_t other = __shfl_sync(0xffffffffu, key, j);
+        if (j < csd) cnt += other < key ? 1 : 0;
+      }
+      if (mine && cnt < k) {
+        L[id] = Lraw + 1;
+        g_sel[td * k + cnt] = (uint8_t)lane;
+      }
+      __syncwarp();
+    }
+    const int32_t* gt = b.gtot + g * E;
+    for (int e = lane; e < E; e += 32) L[e] += gt[e];
+    __syncwarp();
+  }
+}
+
+// Fallback for candidate sets or k wider than a warp, or loads of 2^26 and more: one warp
+// walks every token of the range; 64-bit keys (load, score rank) go through shared memory.
+__device__ __forceinline__ void k2_chain_wide(int32_t* L, unsigned long long* keys,
+                                              const uint16_t* g_cs, const uint8_t* g_ids,
+                                              uint8_t* g_sel, int ntot, int k, int c, int lane) {
+  for (long long t = 0; t < ntot; ++t) {
+    const int cs = g_cs[t];
+    const uint8_t* ids = g_ids + t * c;
+    if (cs <= k) {
+      for (int j = lane; j < k; j += 32) L[ids[j]] += 1;
+    } else {
+      for (int j = lane; j < cs; j += 32)
+        keys[j] = (((unsigned long long)(uint32_t)L[ids[j]]) << 8) | (unsigned)j;
+      __syncwarp();
+      unsigned chosen = 0;
+      int it = 0;
+      for (int j = lane; j < cs; j += 32, ++it) {
+        const unsigned long long key = keys[j];
+        int cnt = 0;
+        for (int i2 = 0; i2 < cs; ++i2) cnt += (keys[i2] < key) ? 1 : 0;
+        if (cnt < k) {
+          g_sel[t * k + cnt] = (uint8_t)j;
+          chosen |= 1u << it;
+        }
+      }
+      __syncwarp();  // loads move only after every lane has finished reading the keys
+      it = 0;
+      for (int j = lane; j < cs; j += 32, ++it)
+        if ((chosen >> it) & 1u) L[ids[j]] += 1;
+    }
+    __syncwarp();
+  }
+}
+
+// Dynamic shared memory: int32 L[E] | uint64 keys[c] | 2 x K2Buffers
+__global__ void __launch_bounds__(kK2Threads) k2_select(const RouteArgs A) {
   extern __shared__ __align__(16) unsigned char k2_smem[];
   const int layer = A.layer0 + blockIdx.x;
-  const int T = A.T, E = A.E, k = A.k, c = A.c;
+  const int E = A.E, k = A.k, c = A.c;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tb = A.tok_begin, ntot = A.tok_end - A.tok_begin;
 
   int32_t* L = reinterpret_cast<int32_t*>(k2_smem);
-  size_t off = align256(sizeof(int32_t) * E);
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(k2_smem + off);
-  off = align256(off + sizeof(unsigned long long) * c);
-  const size_t ids_bytes = align256((size_t)tile_tokens * c);
-  const size_t buf_bytes = ids_bytes + align256(sizeof(uint16_t) * tile_tokens);
-  unsigned char* buf0 = k2_smem + off;
+  unsigned long long* keys =
+      reinterpret_cast<unsigned long long*>(k2_smem + align256(sizeof(int32_t) * E));
+  unsigned char* buf0 = reinterpret_cast<unsigned char*>(keys) +
+                        align256(sizeof(unsigned long long) * c);
+  const size_t buf_bytes = k2_buffer_bytes(E, c);
 
   unsigned char* ws = A.ws + (size_t)layer * A.ws_ls;
-  const uint16_t* g_cs = reinterpret_cast<const uint16_t*>(ws + A.lay.cstar);
-  const uint8_t* g_ids = ws + A.lay.cand_ids;
-  uint8_t* g_sel = ws + A.lay.sel_rank;
+  const uint16_t* g_cs = reinterpret_cast<const uint16_t*>(ws + A.lay.cstar) + tb;
+  const uint8_t* g_ids = ws + A.lay.cand_ids + (size_t)tb * c;
+  uint8_t* g_sel = ws + A.lay.sel_rank + (size_t)tb * k;
   int32_t* g_loads = A.loads + (size_t)layer * E;
-  int32_t* g_eids = A.expert_ids + (size_t)layer * T * k;
 
-  for (int e = tid; e < E; e += kK2Threads) L[e] = g_loads[e];
-  const int n_tiles = (T + tile_tokens - 1) / tile_tokens;
-  if (n_tiles > 0)
-    k2_stage_tile(buf0, reinterpret_cast<uint16_t*>(buf0 + ids_bytes), g_ids, g_cs,
-                  min(tile_tokens, T), c, tid, kK2Threads);
+  int too_big = 0;
+  for (int e = tid; e < E; e += kK2Threads) {
+    const int32_t v = g_loads[e];
+    L[e] = v;
+    // a counter within T of 2^31-1 could wrap during the call: raise the status bit
+    if (v < 0 || v > 0x7fffffff - A.T) { if (A.status) atomicOr(A.status, 1); }
+    if (v < 0 || v > kK2FastMaxLoad - A.T) too_big = 1;
+  }
+  if (__syncthreads_or(too_big) || c > 32 || k > 32) {
+    if (warp == 0) {
+      k2_chain_wide(L, keys, g_cs, g_ids, g_sel, ntot, k, c, lane);
+      for (int e = lane; e < E; e += 32) g_loads[e] = L[e];
+    }
+    return;
+  }
+  const int n_tiles = (ntot + kK2Tile - 1) / kK2Tile;
+
+  auto prep_tile = [&](int tile, int first_warp, int n_warps) {
+    const K2Buffers b = k2_carve(buf0 + (size_t)(tile & 1) * buf_bytes, E, c);
+    const int t0 = tile * kK2Tile;
+    const int ntok = min(kK2Tile, ntot - t0);
+    const int n_groups = (ntok + 31) >> 5;
+    for (int g = warp - first_warp; g < n_groups; g += n_warps)
+      k2_prep_group(b, g, ntok, g_ids + (size_t)t0 * c, g_cs + t0, E, k, c, lane);
+  };
+
+  if (n_tiles > 0) prep_tile(0, 0, kK2Threads / 32);
   __syncthreads();
-
   for (int tile = 0; tile < n_tiles; ++tile) {
-    unsigned char* cur = buf0 + (size_t)(tile & 1) * buf_bytes;
-    unsigned char* nxt = buf0 + (size_t)((tile + 1) & 1) * buf_bytes;
-    const int t0 = tile * tile_tokens;
-    const int ntok = min(tile_tokens, T - t0);
     if (warp > 0) {
-      if (tile + 1 < n_tiles) {
-        const int t1 = t0 + tile_tokens;
-        k2_stage_tile(nxt, reinterpret_cast<uint16_t*>(nxt + ids_bytes), g_ids + (size_t)t1 * c,
-                      g_cs + t1, min(tile_tokens, T - t1), c, tid - 32, kK2Threads - 32);
-      }
+      if (tile + 1 < n_tiles) prep_tile(tile + 1, 1, kK2PrepWarps);
     } else {
-      const uint8_t* s_ids = cur;
-      const uint16_t* s_cs = reinterpret_cast<const uint16_t*>(cur + ids_bytes);
-      for (int i = 0; i < ntok; ++i) {
-        const int cs = s_cs[i];
-        const uint8_t* ids = s_ids + (size_t)i * c;
-        const size_t t = (size_t)(t0 + i);
-        if (cs == 0) {
-          // top-k branch: the choice is already written; only the loads move
-          for (int j = lane; j < k; j += 32) bump_load(L, ids[j], A.status);
-        } else if (cs <= 32) {
-          // one candidate per lane; key = (load, score rank); rank by counting smaller keys
-          const int e = lane < cs ? ids[lane] : 0;
-          const unsigned long long key =
-              lane < cs ? (((unsigned long long)(uint32_t)L[e]) << 8) | (unsigned)lane : ~0ull;
-          int cnt = 0;
-          for (int j = 0; j < cs; ++j) cnt += (__shfl_sync(0xffffffffu, key, j) < key) ? 1 : 0;
-          if (lane < cs && cnt < k) {
-            g_eids[t * k + cnt] = e;
-            g_sel[t * k + cnt] = (uint8_t)lane;
-            bump_load(L, e, A.status);
-          }
-        } else {
-          // wide candidate sets: keys through shared memory, several candidates per lane
-          for (int j = lane; j < cs; j += 32)
-            keys[j] = (((unsigned long long)(uint32_t)L[ids[j]]) << 8) | (unsigned)j;
-          __syncwarp();
-          unsigned chosen = 0;
-          int it = 0;
-          for (int j = lane; j < cs; j += 32, ++it) {
-            const unsigned long long key = keys[j];
-            int cnt = 0;
-            for (int i2 = 0; i2 < cs; ++i2) cnt += (keys[i2] < key) ? 1 : 0;
-            if (cnt < k) {
-              g_eids[t * k + cnt] = ids[j];
-              g_sel[t * k + cnt] = (uint8_t)j;
-              chosen |= 1u << it;
-            }
-          }
-          // loads move only after every lane has finished reading the keys
-          __syncwarp();
-          it = 0;
-          for (int j = lane; j < cs; j += 32, ++it)
-            if ((chosen >> it) & 1u) bump_load(L, ids[j], A.status);
-        }
-        __syncwarp();
-      }
+      const K2Buffers b = k2_carve(buf0 + (size_t)(tile & 1) * buf_bytes, E, c);
+      const int t0 = tile * kK2Tile;
+      const int ntok = min(kK2Tile, ntot - t0);
+      uint8_t* sel = g_sel + (size_t)t0 * k;
+      if (c <= 4) k2_chain_tile<4>(L, b, ntok, E, k, c, sel, lane);
+      else if (c <= 8) k2_chain_tile<8>(L, b, ntok, E, k, c, sel, lane);
+      else if (c <= 16) k2_chain_tile<16>(L, b, ntok, E, k, c, sel, lane);
+      else k2_chain_tile<32>(L, b, ntok, E, k, c, sel, lane);
     }
     __syncthreads();
   }
   for (int e = tid; e < E; e += kK2Threads) g_loads[e] = L[e];
-}
-
-// Combine weights of tokens routed by the load-aware branch: w_j = s[chosen_j], divided by
-// their left-to-right sum when renormalising.  One thread per token.
-__global__ void k2_weights(const RouteArgs A) {
-  const int layer = A.layer0 + blockIdx.y;
-  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= A.T) return;
-  unsigned char* ws = A.ws + (size_t)layer * A.ws_ls;
-  if (reinterpret_cast<const uint16_t*>(ws + A.lay.cstar)[t] == 0) return;
-  const float* sc = reinterpret_cast<const float*>(ws + A.lay.cand_scores) + (size_t)t * A.c;
-  const uint8_t* sel = ws + A.lay.sel_rank + (size_t)t * A.k;
-  float* w = A.weights + ((size_t)layer * A.T + t) * A.k;
-  float sum = 0.0f;
-  for (int j = 0; j < A.k; ++j) {
-    const float v = sc[sel[j]];
-    w[j] = v;
-    sum = j == 0 ? v : __fadd_rn(sum, v);
-  }
-  if (A.renorm)
-    for (int j = 0; j < A.k; ++j) w[j] = __fdiv_rn(w[j], sum);
 }
 
 }  // namespace laser

@@ -3,6 +3,9 @@
 // buffer entry point), no state between calls.
 #include "../../include/laser.h"
 
+#include <cstdlib>
+#include <mutex>
+
 #include "k1_router.cuh"
 #include "k2_select.cuh"
 #include "k3_dispatch.cuh"
@@ -39,7 +42,8 @@ cudaError_t launch_k1(const RouteArgs& a, int n_layers, cudaStream_t s) {
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  dim3 grid((unsigned)((a.T + rows_per_block - 1) / rows_per_block), (unsigned)n_layers);
+  const int ntok = a.tok_end - a.tok_begin;
+  dim3 grid((unsigned)((ntok + rows_per_block - 1) / rows_per_block), (unsigned)n_layers);
   k1_router_mma<NT, MT, KU><<<grid, 128, smem, s>>>(a);
   return cudaGetLastError();
 }
@@ -54,14 +58,54 @@ cudaError_t launch_k1_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   return launch_k1<32, 1, 1>(a, n_layers, s);
 }
 
-int k2_tile_tokens(int c) { return c <= 128 ? 128 : 64; }
+size_t k2_smem_bytes(int E, int c, int k) {
+  const size_t base = align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c);
+  if (c > 32 || k > 32) return base;  // wide fallback: no staged tiles
+  return base + 2 * k2_buffer_bytes(E, c);
+}
 
-size_t k2_smem_bytes(int E, int c) {
-  const int tile = k2_tile_tokens(c);
-  size_t off = align256(sizeof(int32_t) * E);
-  off = align256(off + sizeof(unsigned long long) * c);
-  const size_t buf = align256((size_t)tile * c) + align256(sizeof(uint16_t) * tile);
-  return off + 2 * buf;
+// Per-device helper objects for overlapping the ordered selection of one token chunk with
+// the router kernel of the next: one high-priority side stream and a few events, created on
+// first use and kept until the process exits.
+constexpr int kMaxChunks = 16;
+struct DeviceAux {
+  bool ready = false;
+  cudaStream_t side = nullptr;
+  cudaEvent_t k1_done[kMaxChunks] = {};
+  cudaEvent_t side_done = nullptr;
+};
+DeviceAux g_aux[64];
+std::mutex g_aux_mutex;
+
+DeviceAux* get_aux() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  DeviceAux& a = g_aux[dev];
+  if (!a.ready) {
+    int lo = 0, hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&a.side, cudaStreamNonBlocking, hi) != cudaSuccess)
+      return nullptr;
+    for (int i = 0; i < kMaxChunks; ++i)
+      if (cudaEventCreateWithFlags(&a.k1_done[i], cudaEventDisableTiming) != cudaSuccess)
+        return nullptr;
+    if (cudaEventCreateWithFlags(&a.side_done, cudaEventDisableTiming) != cudaSuccess)
+      return nullptr;
+    a.ready = true;
+  }
+  return &a;
+}
+
+// Tokens per chunk of the router/selection pipeline (multiple of the selection tile).
+int chunk_tokens(int T) {
+  static const int env = [] {
+    const char* v = std::getenv("LASER_CHUNK_TOKENS");
+    return v ? std::atoi(v) : 0;
+  }();
+  int ct = env > 0 ? env : 4096;
+  ct = ((ct + kK2Tile - 1) / kK2Tile) * kK2Tile;
+  while ((T + ct - 1) / ct > kMaxChunks) ct *= 2;
+  return ct;
 }
 
 // Enqueues all stages for layers [layer0, layer0 + n) of a batched call.
@@ -78,19 +122,39 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   cudaError_t e = cudaSuccess;
   if (!mark(0)) return LASER_ERR_CUDA;
   if (a.T > 0) {
-    e = launch_k1_for_E(a, n, s);
-    if (e != cudaSuccess) return LASER_ERR_CUDA;
-    if (!mark(1)) return LASER_ERR_CUDA;
-    const size_t smem2 = k2_smem_bytes(a.E, a.c);
+    const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
     if (smem2 > 48 * 1024) {
       e = cudaFuncSetAttribute(k2_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
       if (e != cudaSuccess) return LASER_ERR_CUDA;
     }
-    k2_select<<<n, kK2Threads, smem2, s>>>(a, k2_tile_tokens(a.c));
-    if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-    dim3 gw((unsigned)((a.T + 255) / 256), (unsigned)n);
-    k2_weights<<<gw, 256, 0, s>>>(a);
-    if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+    const int ct = chunk_tokens(a.T);
+    const int n_chunks = (a.T + ct - 1) / ct;
+    if (n_chunks == 1) {
+      a.tok_begin = 0; a.tok_end = a.T;
+      if (launch_k1_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
+      if (!mark(1)) return LASER_ERR_CUDA;
+      k2_select<<<n, kK2Threads, smem2, s>>>(a);
+      if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+    } else {
+      // router kernel of chunk i+1 on the caller's stream overlaps the selection of chunk i
+      // on the side stream; the selection kernels run in chunk order and carry the loads
+      std::lock_guard<std::mutex> lock(g_aux_mutex);
+      DeviceAux* aux = get_aux();
+      if (!aux) return LASER_ERR_CUDA;
+      for (int ch = 0; ch < n_chunks; ++ch) {
+        a.tok_begin = ch * ct;
+        a.tok_end = a.tok_begin + ct < a.T ? a.tok_begin + ct : a.T;
+        if (launch_k1_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
+        if (cudaEventRecord(aux->k1_done[ch], s) != cudaSuccess) return LASER_ERR_CUDA;
+        if (cudaStreamWaitEvent(aux->side, aux->k1_done[ch], 0) != cudaSuccess)
+          return LASER_ERR_CUDA;
+        k2_select<<<n, kK2Threads, smem2, aux->side>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+      }
+      if (!mark(1)) return LASER_ERR_CUDA;
+      if (cudaEventRecord(aux->side_done, aux->side) != cudaSuccess) return LASER_ERR_CUDA;
+      if (cudaStreamWaitEvent(s, aux->side_done, 0) != cudaSuccess) return LASER_ERR_CUDA;
+    }
   } else if (!mark(1)) {
     return LASER_ERR_CUDA;
   }
@@ -101,8 +165,13 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
   k3_scan<<<n, kK3Threads, 0, s>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-  k3_scatter<<<g3, kK3Threads, smem3, s>>>(a);
+  k3_rank<<<g3, kK3Threads, smem3, s>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+  if (a.T > 0) {
+    dim3 gf((unsigned)((a.T + 127) / 128), (unsigned)n);
+    k3_finalize<<<gf, 128, 0, s>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
+  }
   if (!mark(3)) return LASER_ERR_CUDA;
   return LASER_OK;
 }

@@ -14,6 +14,7 @@ struct WorkspaceLayout {
   size_t cand_ids;     // uint8  [T, c]     ranking pi(0..c-1)
   size_t cand_scores;  // float  [T, c]     s_pi(j)
   size_t sel_rank;     // uint8  [T, k]     rank positions chosen by the load-aware scan
+  size_t pair_dst;     // int32  [T*k]      destination index in perm of pair t*k+j (score order)
   size_t blk_hist;     // int32  [n_blk, E] dispatch block histograms, then block bases
   size_t total;        // bytes per layer, multiple of 256
   int n_blk;           // dispatch blocks per layer
@@ -30,6 +31,7 @@ inline WorkspaceLayout make_layout(int T, int E, int k, int c) {
   w.cand_ids = off;     off = align256(off + (size_t)T * c);
   w.cand_scores = off;  off = align256(off + sizeof(float) * (size_t)T * c);
   w.sel_rank = off;     off = align256(off + (size_t)T * k);
+  w.pair_dst = off;     off = align256(off + sizeof(int32_t) * (size_t)T * k);
   long long pairs = (long long)T * k;
   w.n_blk = (int)((pairs + kDispatchPairsPerBlock - 1) / kDispatchPairsPerBlock);
   if (w.n_blk < 1) w.n_blk = 1;
@@ -57,9 +59,18 @@ struct RouteArgs {
   int T, d, E, k, c, n_bins, renorm;
   long long ld_h, ld_w;
   int layer0;              // first layer of this launch
+  int tok_begin, tok_end;  // token range of this launch (router and selection kernels)
   float eps_high[kMaxLayersPerLaunch];
   float t_fix[kMaxLayersPerLaunch];
 };
+
+// Rank position (in the score ranking) of slot j of token t as the selection left it:
+// tokens with c* > k were decided by the load-aware scan (sel_rank), all others keep their
+// k best in score order.
+__device__ __forceinline__ int pair_rank(const uint16_t* cstar, const uint8_t* sel_rank, int k,
+                                         long long t, int j) {
+  return cstar[t] > k ? sel_rank[t * k + j] : j;
+}
 
 // fp32 exponential for y <= 0 with a fixed sequence of correctly rounded operations:
 //   y < -80 -> 0;  n = rint(y*log2e);  r = y - n*ln2 (two fma steps);
