@@ -5,15 +5,22 @@
 // Only tokens whose candidate set is larger than k (c* > k, "decision tokens") have a
 // load-dependent choice.  Every other token (top-k branch, or c* == k) sends its k best
 // experts whatever the loads are, so its increments are known without the chain.  The block
-// therefore splits the work:
-//   prep warps   stage a tile of candidate records in shared memory and, per group of 32
-//                tokens, count the fixed increments per expert (group totals) and, for every
-//                candidate of every decision token, the fixed increments of earlier tokens
-//                of the same group (ballot + popcount);
-//   chain warp   walks the decision tokens only: load seen by candidate j =
-//                L[e_j] (all earlier groups + earlier decisions) + its in-group prefix;
-//                ranks the candidates by (load, score rank) with warp shuffles, bumps the
-//                k winners, and adds the group totals at each group end.
+// therefore splits the work, tile by tile (double buffered in shared memory):
+//   prep warps   stage the candidate records (cp.async), count the fixed increments per group
+//                of 32 tokens, prefix them over the tile, and write a dense, ordered list of
+//                the tile's decision tokens.  A list entry holds one word per lane of the
+//                chain warp with the addend (fixed increments seen so far in the tile << 5 |
+//                score rank), so that a candidate's key is
+//                    (load at tile start + decisions so far) << 5 + addend.
+//   chain warp   walks the list with the next entry prefetched into registers; per entry it
+//                forms the keys, ranks each candidate by counting smaller keys (one shuffle
+//                per candidate), bumps the k winners and records their score ranks.
+// A single warp is a slow sequential machine (a dependent instruction issues every few
+// cycles), so everything that does not depend on the loads is moved into the prep warps and
+// the chain loop is kept to a few dozen instructions.
+// Two chain layouts:
+//   E <= 32, c <= 16   lane = expert, loads stay in a register of the chain warp;
+//   otherwise          lane = candidate, loads in shared memory.
 // The slot order of c* == k tokens, which depends on the loads they saw, is reconstructed
 // afterwards from the dispatch ranks (k3_finalize).
 #pragma once
@@ -22,120 +29,249 @@
 namespace laser {
 
 constexpr int kK2Threads = 256;
-constexpr int kK2PrepWarps = kK2Threads / 32 - 1;
-constexpr int kK2Tile = 256;             // tokens per shared-memory buffer
-constexpr int kK2Groups = kK2Tile / 32;
-constexpr int kK2FastMaxLoad = 1 << 26;  // 32-bit keys (load << 5 | rank) need loads below this
+constexpr int kK2Warps = kK2Threads / 32;
+constexpr int kK2MaxTile = 512;          // tokens per buffer: 512 (lane = expert) or 256
+constexpr int kK2MaxGroups = kK2MaxTile / 32;
+constexpr int kK2FastMaxLoad = 1 << 25;  // 32-bit keys (load << 5 | rank) stay below 2^31
+constexpr int kK2EntryWords = 40;        // 32 lane words | 4 words of source lanes | sel base
+constexpr uint32_t kK2NoCand = 0x80000000u;
+
+__host__ __device__ inline int k2_tile_tokens(int E, int c) { return (E <= 32 && c <= 16) ? 512 : 256; }
 
 struct K2Buffers {
-  uint8_t* ids;     // [kK2Tile * c] ranked candidate ids
-  uint8_t* pre;     // [kK2Tile * c] in-group fixed increments seen by each candidate
-  uint16_t* cs;     // [kK2Tile]
-  int32_t* gtot;    // [kK2Groups * E] fixed increments per group and expert
+  uint8_t* ids;     // [tile * c]         staged ranked candidate ids
+  uint16_t* cs;     // [tile]             staged c*
+  uint32_t* gB;     // [groups * 32]      E <= 32: per group and expert, ballot of fixed senders
+  int32_t* gtot;    // [groups * max(E,32)] fixed increments per group and expert, then their
+                    //                    exclusive prefix over the groups of the tile
+  int32_t* ttot;    // [max(E,32)]        fixed increments of the whole tile per expert
+  int32_t* dcount;  // [kK2MaxGroups]     decision tokens per group
+  uint32_t* list;   // [(tile + 1) * kK2EntryWords] decision-token entries
 };
 
 __host__ __device__ inline size_t k2_buffer_bytes(int E, int c) {
-  return 2 * align256((size_t)kK2Tile * c) + align256(sizeof(uint16_t) * kK2Tile) +
-         align256(sizeof(int32_t) * kK2Groups * E);
+  const int tile = k2_tile_tokens(E, c), groups = tile / 32, Ew = E > 32 ? E : 32;
+  return align256((size_t)tile * c) + align256(sizeof(uint16_t) * tile) +
+         align256(sizeof(uint32_t) * groups * 32) + align256(sizeof(int32_t) * groups * Ew) +
+         align256(sizeof(int32_t) * Ew) + align256(sizeof(int32_t) * kK2MaxGroups) +
+         align256(sizeof(uint32_t) * (tile + 1) * kK2EntryWords);
 }
 
-__device__ __forceinline__ K2Buffers k2_carve(unsigned char* base, int E, int c) {
+__device__ __forceinline__ K2Buffers k2_carve(unsigned char* p, int E, int c) {
+  const int tile = k2_tile_tokens(E, c), groups = tile / 32, Ew = E > 32 ? E : 32;
   K2Buffers b;
-  b.ids = base;
-  b.pre = base + align256((size_t)kK2Tile * c);
-  b.cs = reinterpret_cast<uint16_t*>(base + 2 * align256((size_t)kK2Tile * c));
-  b.gtot = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(b.cs) +
-                                      align256(sizeof(uint16_t) * kK2Tile));
+  b.ids = p;                                 p += align256((size_t)tile * c);
+  b.cs = reinterpret_cast<uint16_t*>(p);     p += align256(sizeof(uint16_t) * tile);
+  b.gB = reinterpret_cast<uint32_t*>(p);     p += align256(sizeof(uint32_t) * groups * 32);
+  b.gtot = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * groups * Ew);
+  b.ttot = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * Ew);
+  b.dcount = reinterpret_cast<int32_t*>(p);  p += align256(sizeof(int32_t) * kK2MaxGroups);
+  b.list = reinterpret_cast<uint32_t*>(p);
   return b;
 }
 
-// Prepares one group of 32 tokens (lane = token) of a tile.
-__device__ __forceinline__ void k2_prep_group(const K2Buffers& b, int g, int ntok,
-                                              const uint8_t* g_ids, const uint16_t* g_cs, int E,
-                                              int k, int c, int lane) {
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src));
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.wait_all;" ::: "memory");
+}
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Issues the copies of one group's records (32 tokens) into the tile buffer.
+__device__ __forceinline__ void k2_stage_group(const K2Buffers& b, int g, int ntok,
+                                               const uint8_t* g_ids, const uint16_t* g_cs, int c,
+                                               int lane) {
+  const int n_here = min(32, ntok - g * 32);
+  const uint8_t* src = g_ids + (size_t)g * 32 * c;
+  uint8_t* dst = b.ids + g * 32 * c;
+  if (n_here == 32) {
+    for (int i = lane; i < 2 * c; i += 32) cp_async16(dst + 16 * i, src + 16 * i);
+    if (lane < 4) cp_async16(b.cs + g * 32 + lane * 8, g_cs + g * 32 + lane * 8);
+  } else {
+    for (int i = lane; i < n_here * c; i += 32) dst[i] = src[i];
+    b.cs[g * 32 + lane] = lane < n_here ? g_cs[g * 32 + lane] : (uint16_t)0;
+  }
+}
+
+// Phase 1 for one staged group (lane = token): decision count and the fixed increments.
+__device__ __forceinline__ void k2_count_group(const K2Buffers& b, int g, int ntok, int E, int Ew,
+                                               int k, int c, bool small_e, int lane) {
   const int tok = g * 32 + lane;
   const bool valid = tok < ntok;
-  const int n_here = min(32, ntok - g * 32);
-  // stage this group's records
-  {
-    const int bytes = n_here * c;
-    const uint8_t* src = g_ids + (size_t)g * 32 * c;
-    uint8_t* dst = b.ids + (size_t)g * 32 * c;
-    const int n16 = bytes >> 4;
-    for (int i = lane; i < n16; i += 32)
-      reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
-    for (int i = (n16 << 4) + lane; i < bytes; i += 32) dst[i] = src[i];
-  }
-  const int cs = valid ? g_cs[tok] : 0;
-  b.cs[tok] = (uint16_t)cs;
-  int32_t* gt = b.gtot + g * E;
-  for (int e = lane; e < E; e += 32) gt[e] = 0;
-  __syncwarp();
+  const int cs = valid ? b.cs[tok] : 0;
   const bool fixed = valid && cs <= k;
-  const uint8_t* my = b.ids + (size_t)tok * c;
-  if (fixed)
-    for (int j = 0; j < k; ++j) atomicAdd(&gt[my[j]], 1);
-  unsigned dmask = __ballot_sync(0xffffffffu, valid && cs > k);
-  while (dmask) {
-    const int dl = __ffs(dmask) - 1;
-    dmask &= dmask - 1;
-    const int csd = __shfl_sync(0xffffffffu, cs, dl);
-    const uint8_t* cand = b.ids + (size_t)(g * 32 + dl) * c;
+  const uint8_t* my = b.ids + tok * c;
+  const unsigned dmask = __ballot_sync(0xffffffffu, valid && cs > k);
+  if (lane == 0) b.dcount[g] = __popc(dmask);
+  if (small_e) {
+    uint32_t m = 0;
+    if (fixed)
+      for (int j = 0; j < k; ++j) m |= 1u << my[j];
+    uint32_t mineB = 0;
+    for (int e = 0; e < E; ++e) {
+      const uint32_t B = __ballot_sync(0xffffffffu, (m >> e) & 1u);
+      if (lane == e) mineB = B;
+    }
+    b.gB[g * 32 + lane] = mineB;
+  } else {
+    int32_t* gt = b.gtot + g * Ew;
+    for (int e = lane; e < E; e += 32) gt[e] = 0;
+    __syncwarp();
+    if (fixed)
+      for (int j = 0; j < k; ++j) atomicAdd(&gt[my[j]], 1);
+  }
+}
+
+// Phase 2 for one group: appends its decision tokens to the tile's list.
+template <int KREG>
+__device__ __forceinline__ void k2_list_group(const K2Buffers& b, int g, int ntok, int E, int Ew,
+                                              int k, int c, bool small_e, int lane) {
+  const int tok = g * 32 + lane;
+  const bool valid = tok < ntok;
+  const int cs = valid ? b.cs[tok] : 0;
+  const uint8_t* my = b.ids + tok * c;
+  const bool dec = valid && cs > k;
+  const unsigned dmask = __ballot_sync(0xffffffffu, dec);
+  if (dmask == 0) return;
+  int dbase = 0;
+  for (int g2 = 0; g2 < g; ++g2) dbase += b.dcount[g2];
+  const int nd = __popc(dmask);
+  const unsigned below = (1u << lane) - 1;
+  const int32_t* gpre = b.gtot + g * Ew;   // fixed increments in earlier groups of the tile
+
+  if (small_e) {
+    // lane = decision token builds its own entry (lane words indexed by expert)
+    uint32_t* ent0 = b.list + dbase * kK2EntryWords;
+    for (int i = lane; i < nd * 32; i += 32) ent0[(i >> 5) * kK2EntryWords + (i & 31)] = kK2NoCand;
+    __syncwarp();
+    if (dec) {
+      uint32_t* ent = ent0 + __popc(dmask & below) * kK2EntryWords;
+      const uint32_t* B = b.gB + g * 32;
+      uint32_t cmask = 0;
+      for (int r = 0; r < cs; ++r) {
+        const int e = my[r];
+        cmask |= 1u << e;
+        ent[e] = ((uint32_t)(gpre[e] + __popc(B[e] & below)) << 5) | (uint32_t)r;
+      }
+      const uint32_t pad = (uint32_t)(__ffs(~cmask) - 1);   // a lane that holds no candidate
+      uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t v = j < cs ? (uint32_t)my[j] : pad;
+        w[j >> 2] |= v << (8 * (j & 3));
+      }
+      ent[32] = w[0]; ent[33] = w[1]; ent[34] = w[2]; ent[35] = w[3];
+      ent[36] = (uint32_t)(tok * k);
+    }
+    return;
+  }
+
+  // lane = candidate: one decision token after the other, one ballot per candidate
+  const bool fixed = valid && cs <= k;
+  int myid[KREG > 0 ? KREG : 1];
+#pragma unroll
+  for (int j = 0; j < KREG; ++j) myid[j] = (fixed && j < k) ? my[j] : -1;
+  unsigned rest = dmask;
+  while (rest) {
+    const int dl = __ffs(rest) - 1;
+    rest &= rest - 1;
     const unsigned before = (1u << dl) - 1;
+    uint32_t* ent = b.list + (dbase + __popc(dmask & before)) * kK2EntryWords;
+    const int csd = __shfl_sync(0xffffffffu, cs, dl);
+    const uint8_t* cand = b.ids + (g * 32 + dl) * c;
     int mine = 0;
-    for (int r = 0; r < csd; ++r) {
+    for (int r = 0; r < csd; ++r) {   // csd <= 32 on this path
       const int e = cand[r];
       bool hit = false;
-      if (fixed)
+      if (KREG > 0) {
+#pragma unroll
+        for (int j = 0; j < KREG; ++j) hit |= (myid[j] == e);
+      } else if (fixed) {
         for (int j = 0; j < k; ++j) hit |= (my[j] == e);
-      const int cnt = __popc(__ballot_sync(0xffffffffu, hit) & before);
-      if (lane == (r & 31)) mine = cnt;
-      if ((r & 31) == 31 || r == csd - 1) {
-        const int rr = (r & ~31) + lane;
-        if (rr <= r) b.pre[(size_t)(g * 32 + dl) * c + rr] = (uint8_t)mine;
       }
+      const int cnt = __popc(__ballot_sync(0xffffffffu, hit) & before);
+      if (lane == r) mine = cnt;
+    }
+    uint32_t word = 0x8000u;
+    if (lane < csd) {
+      const int e = cand[lane];
+      word = ((uint32_t)(mine + gpre[e]) << 5) | (uint32_t)lane | ((uint32_t)e << 16);
+    }
+    ent[lane] = word;
+    if (lane == 0) ent[36] = (uint32_t)((g * 32 + dl) * k);
+  }
+}
+
+// Chain over one tile's list, lane = expert.  Le32 = (load of expert `lane`) << 5.
+template <int CMAX>
+__device__ __forceinline__ void k2_chain_experts(uint32_t& Le32, const uint32_t* list, int n_dec,
+                                                 int k, uint8_t* sel, int lane) {
+  constexpr int SW = (CMAX + 3) / 4;
+  uint32_t add_n = list[lane], base_n = list[36];
+  uint32_t src_n[SW];
+#pragma unroll
+  for (int q = 0; q < SW; ++q) src_n[q] = list[32 + q];
+#pragma unroll 1
+  for (int i = 0; i < n_dec; ++i) {
+    const uint32_t add = add_n, base = base_n;
+    uint32_t src[SW];
+#pragma unroll
+    for (int q = 0; q < SW; ++q) src[q] = src_n[q];
+    const uint32_t* nx = list + (i + 1) * kK2EntryWords;   // the list has one spare entry
+    add_n = nx[lane];
+    base_n = nx[36];
+#pragma unroll
+    for (int q = 0; q < SW; ++q) src_n[q] = nx[32 + q];
+    const uint32_t key = Le32 + add;
+    // all shuffles are issued before the first compare, so their latencies overlap
+    uint32_t other[CMAX];
+#pragma unroll
+    for (int j = 0; j < CMAX; ++j)
+      other[j] = __shfl_sync(0xffffffffu, key, (int)(src[j >> 2] >> (8 * (j & 3))));
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < CMAX; ++j) cnt += other[j] < key ? 1 : 0;
+    if (cnt < k && (int32_t)key >= 0) {
+      Le32 += 32;
+      sel[base + cnt] = (uint8_t)(add & 31u);
     }
   }
 }
 
-// Chain over one tile, candidate sets no wider than a warp, loads below 2^26.
+// Chain over one tile's list, lane = candidate, loads in shared memory.
 template <int CMAX>
-__device__ __forceinline__ void k2_chain_tile(int32_t* L, const K2Buffers& b, int ntok, int E,
-                                              int k, int c, uint8_t* g_sel, int lane) {
-  const int n_groups = (ntok + 31) >> 5;
-  for (int g = 0; g < n_groups; ++g) {
-    const int tok = g * 32 + lane;
-    const int cs_l = tok < ntok ? b.cs[tok] : 0;
-    unsigned dmask = __ballot_sync(0xffffffffu, cs_l > k);
-    while (dmask) {
-      const int dl = __ffs(dmask) - 1;
-      dmask &= dmask - 1;
-      const int csd = __shfl_sync(0xffffffffu, cs_l, dl);
-      const size_t td = (size_t)(g * 32 + dl);
-      const bool mine = lane < csd;
-      const int id = mine ? b.ids[td * c + lane] : 0;
-      const int p = mine ? b.pre[td * c + lane] : 0;
-      const int32_t Lraw = mine ? L[id] : 0;
-      const uint32_t key = mine ? (((uint32_t)(Lraw + p) << 5) | (uint32_t)lane) : 0xffffffffu;
-      int cnt = 0;
+__device__ __forceinline__ void k2_chain_cands(int32_t* L, const uint32_t* list, int n_dec, int k,
+                                               uint8_t* sel, int lane) {
+  uint32_t w_n = list[lane], base_n = list[36];
+#pragma unroll 1
+  for (int i = 0; i < n_dec; ++i) {
+    const uint32_t w = w_n, base = base_n;
+    const uint32_t* nx = list + (i + 1) * kK2EntryWords;   // the list has one spare entry
+    w_n = nx[lane];
+    base_n = nx[36];
+    const bool cand = (w & 0x8000u) == 0;
+    const int id = (int)(w >> 16);
+    const int32_t Lraw = L[id];
+    const uint32_t key = cand ? ((uint32_t)Lraw << 5) + (w & 0x7fffu) : 0xffffffffu;
+    uint32_t other[CMAX];
 #pragma unroll
-      for (int j = 0; j < CMAX; ++j) {
-        const uint32_t other = __shfl_sync(0xffffffffu, key, j);
-        if (j < csd) cnt += other < key ? 1 : 0;
-      }
-      if (mine && cnt < k) {
-        L[id] = Lraw + 1;
-        g_sel[td * k + cnt] = (uint8_t)lane;
-      }
-      __syncwarp();
+    for (int j = 0; j < CMAX; ++j) other[j] = __shfl_sync(0xffffffffu, key, j);
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < CMAX; ++j) cnt += other[j] < key ? 1 : 0;
+    if (cand && cnt < k) {
+      L[id] = Lraw + 1;
+      sel[base + cnt] = (uint8_t)lane;
     }
-    const int32_t* gt = b.gtot + g * E;
-    for (int e = lane; e < E; e += 32) L[e] += gt[e];
     __syncwarp();
   }
 }
 
-// Fallback for candidate sets or k wider than a warp, or loads of 2^26 and more: one warp
+// Fallback for candidate sets or k wider than a warp, or loads of 2^25 and more: one warp
 // walks every token of the range; 64-bit keys (load, score rank) go through shared memory.
 __device__ __forceinline__ void k2_chain_wide(int32_t* L, unsigned long long* keys,
                                               const uint16_t* g_cs, const uint8_t* g_ids,
@@ -205,35 +341,76 @@ __global__ void __launch_bounds__(kK2Threads) k2_select(const RouteArgs A) {
     }
     return;
   }
-  const int n_tiles = (ntot + kK2Tile - 1) / kK2Tile;
+  const bool small_e = E <= 32 && c <= 16;
+  const int tile_tokens = k2_tile_tokens(E, c);
+  const int Ew = E > 32 ? E : 32;
+  const int n_tiles = (ntot + tile_tokens - 1) / tile_tokens;
 
-  auto prep_tile = [&](int tile, int first_warp, int n_warps) {
+  // Tile preparation by warps [first_warp, first_warp + n_warps); bar_id names their barrier.
+  auto prep_tile = [&](int tile, int first_warp, int n_warps, int bar_id) {
     const K2Buffers b = k2_carve(buf0 + (size_t)(tile & 1) * buf_bytes, E, c);
-    const int t0 = tile * kK2Tile;
-    const int ntok = min(kK2Tile, ntot - t0);
+    const int t0 = tile * tile_tokens;
+    const int ntok = min(tile_tokens, ntot - t0);
     const int n_groups = (ntok + 31) >> 5;
-    for (int g = warp - first_warp; g < n_groups; g += n_warps)
-      k2_prep_group(b, g, ntok, g_ids + (size_t)t0 * c, g_cs + t0, E, k, c, lane);
+    const int w = warp - first_warp;
+    for (int g = w; g < n_groups; g += n_warps)
+      k2_stage_group(b, g, ntok, g_ids + (size_t)t0 * c, g_cs + t0, c, lane);
+    cp_async_wait_all();
+    __syncwarp();
+    for (int g = w; g < n_groups; g += n_warps)
+      k2_count_group(b, g, ntok, E, Ew, k, c, small_e, lane);
+    for (int g = n_groups + w; g < kK2MaxGroups; g += n_warps)
+      if (lane == 0) b.dcount[g] = 0;
+    named_barrier(bar_id, n_warps * 32);
+    // exclusive prefix of the fixed increments over the groups, and the tile totals
+    for (int e = w * 32 + lane; e < E; e += n_warps * 32) {
+      int32_t run = 0;
+      for (int g = 0; g < n_groups; ++g) {
+        const int32_t v = small_e ? __popc(b.gB[g * 32 + e]) : b.gtot[g * Ew + e];
+        b.gtot[g * Ew + e] = run;
+        run += v;
+      }
+      b.ttot[e] = run;
+    }
+    named_barrier(bar_id, n_warps * 32);
+    for (int g = w; g < n_groups; g += n_warps) {
+      if (k <= 8) k2_list_group<8>(b, g, ntok, E, Ew, k, c, small_e, lane);
+      else k2_list_group<0>(b, g, ntok, E, Ew, k, c, small_e, lane);
+    }
   };
 
-  if (n_tiles > 0) prep_tile(0, 0, kK2Threads / 32);
+  if (n_tiles > 0) prep_tile(0, 0, kK2Warps, 1);
   __syncthreads();
+  uint32_t Le32 = (warp == 0 && lane < E) ? (uint32_t)L[lane] << 5 : 0;
   for (int tile = 0; tile < n_tiles; ++tile) {
     if (warp > 0) {
-      if (tile + 1 < n_tiles) prep_tile(tile + 1, 1, kK2PrepWarps);
+      if (tile + 1 < n_tiles) prep_tile(tile + 1, 1, kK2Warps - 1, 2);
     } else {
       const K2Buffers b = k2_carve(buf0 + (size_t)(tile & 1) * buf_bytes, E, c);
-      const int t0 = tile * kK2Tile;
-      const int ntok = min(kK2Tile, ntot - t0);
-      uint8_t* sel = g_sel + (size_t)t0 * k;
-      if (c <= 4) k2_chain_tile<4>(L, b, ntok, E, k, c, sel, lane);
-      else if (c <= 8) k2_chain_tile<8>(L, b, ntok, E, k, c, sel, lane);
-      else if (c <= 16) k2_chain_tile<16>(L, b, ntok, E, k, c, sel, lane);
-      else k2_chain_tile<32>(L, b, ntok, E, k, c, sel, lane);
+      uint8_t* sel = g_sel + (size_t)tile * tile_tokens * k;
+      int n_dec = lane < kK2MaxGroups ? b.dcount[lane] : 0;
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) n_dec += __shfl_xor_sync(0xffffffffu, n_dec, s);
+      if (small_e) {
+        if (c <= 4) k2_chain_experts<4>(Le32, b.list, n_dec, k, sel, lane);
+        else if (c <= 8) k2_chain_experts<8>(Le32, b.list, n_dec, k, sel, lane);
+        else k2_chain_experts<16>(Le32, b.list, n_dec, k, sel, lane);
+        if (lane < E) Le32 += (uint32_t)b.ttot[lane] << 5;
+      } else {
+        if (c <= 8) k2_chain_cands<8>(L, b.list, n_dec, k, sel, lane);
+        else if (c <= 16) k2_chain_cands<16>(L, b.list, n_dec, k, sel, lane);
+        else k2_chain_cands<32>(L, b.list, n_dec, k, sel, lane);
+        for (int e = lane; e < E; e += 32) L[e] += b.ttot[e];
+        __syncwarp();
+      }
     }
     __syncthreads();
   }
-  for (int e = tid; e < E; e += kK2Threads) g_loads[e] = L[e];
+  if (small_e) {
+    if (warp == 0 && lane < E) g_loads[lane] = (int32_t)(Le32 >> 5);
+  } else {
+    for (int e = tid; e < E; e += kK2Threads) g_loads[e] = L[e];
+  }
 }
 
 }  // namespace laser

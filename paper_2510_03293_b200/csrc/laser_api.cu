@@ -103,7 +103,7 @@ int chunk_tokens(int T) {
     return v ? std::atoi(v) : 0;
   }();
   int ct = env > 0 ? env : 4096;
-  ct = ((ct + kK2Tile - 1) / kK2Tile) * kK2Tile;
+  ct = ((ct + kK2MaxTile - 1) / kK2MaxTile) * kK2MaxTile;
   while ((T + ct - 1) / ct > kMaxChunks) ct *= 2;
   return ct;
 }
