@@ -52,15 +52,9 @@ def workload_config(w, n_layers):
 
 
 def launches_per_step(w, L) -> int:
-    """Kernels the library enqueues per step: router + selection per token chunk, then the
-    four dispatch kernels, per group of at most 64 layers."""
-    chunk = int(os.environ.get("LASER_CHUNK_TOKENS", "4096") or 4096)
-    chunk = -(-chunk // 256) * 256
-    n_chunks = -(-w.T // chunk)
-    while n_chunks > 16:
-        chunk *= 2
-        n_chunks = -(-w.T // chunk)
-    return (2 * n_chunks + 4) * ((L + 63) // 64)
+    """Kernels the library enqueues per step, per group of at most 64 layers: the fused
+    router + selection kernel and the four dispatch kernels."""
+    return 5 * ((L + 63) // 64)
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
@@ -231,7 +225,6 @@ def run_gpu(args, w):
     value = world * tokens / (ms_per_step * 1e-3)
 
     k1 = sum(ev[0].elapsed_time(ev[1]) for ev in stage) / args.steps
-    k2 = sum(ev[1].elapsed_time(ev[2]) for ev in stage) / args.steps
     k3 = sum(ev[2].elapsed_time(ev[3]) for ev in stage) / args.steps
     peak, peak_kind = measured_peak_hbm()
     bytes_per_launch = algorithmic_bytes_per_token(w) * tokens
@@ -247,11 +240,11 @@ def run_gpu(args, w):
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate and scores",
         "data": "synthetic", "config": workload_config(w, L),
-        "roofline": {"bound": "hbm", "kernel": "k1_router_mma (contraction + score epilogue)",
+        "roofline": {"bound": "hbm", "kernel": "k12_route_select (contraction + score epilogue + ordered selection)",
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": None,
                      "bytes_per_launch": bytes_per_launch},
-        "path": {"k1_ms": k1, "k2_ms": k2, "k3_ms": k3, "path_gbs": path_gbs,
+        "path": {"router_select_ms": k1, "dispatch_ms": k3, "path_gbs": path_gbs,
                  "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
         "routing": {"mean_imbalance_max_over_mean": imb, "status_word": status},
         "gpu_launches": launches_per_step(w, L) * args.steps,

@@ -19,16 +19,11 @@
  *   - The caller owns every buffer; no routing state is kept between calls.
  *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*); the call
  *     returns without synchronising, except laser_route_host, which synchronises the stream
- *     before returning.  Calls with more tokens than one chunk (4096 by default, environment
- *     variable LASER_CHUNK_TOKENS) overlap the ordered selection of one chunk with the router
- *     kernel of the next on a library-owned high-priority side stream; that stream and a few
- *     events are created per device on the first such call and live until the process
- *     exits.  The side work is joined back into the caller's stream before the call's last
- *     kernels, so stream order as seen by the caller is unchanged.
+ *     before returning.
  *   - Return value: LASER_OK (0) or a negative status.  On a validation error nothing is
  *     launched and no output is touched.
  *   - Conditions only visible on the device are OR-ed into *status_word (device int32,
- *     may be NULL): LASER_DEV_LOAD_OVERFLOW.
+ *     may be NULL): LASER_DEV_LOAD_OVERFLOW, LASER_DEV_TIMEOUT.
  */
 #ifndef LASER_H_
 #define LASER_H_
@@ -49,9 +44,13 @@ enum {
   LASER_ERR_CUDA = -5              /* a CUDA runtime call failed (launch error) */
 };
 
-/* Bit in *status_word: on entry some load counter was negative or within T of 2^31-1, so it
- * could overflow during the call; the call's results are then unspecified. */
-enum { LASER_DEV_LOAD_OVERFLOW = 1 };
+/* Bits in *status_word.
+ * LOAD_OVERFLOW: on entry some load counter was negative or within T of 2^31-1, so it could
+ *   overflow during the call.
+ * TIMEOUT: the ordered selection runs in the same launch as the router and waits for the
+ *   router's tiles; a wait gave up after about two seconds (it never should).
+ * When either bit is set the call's results are unspecified. */
+enum { LASER_DEV_LOAD_OVERFLOW = 1, LASER_DEV_TIMEOUT = 2 };
 
 enum { LASER_MAX_EXPERTS = 256 };
 
@@ -149,10 +148,11 @@ int laser_route_layers(int32_t n_layers,
 
 /*
  * laser_route_layers that also records CUDA events between its stages, so that a caller can
- * time the router contraction (stage 1-4), the ordered selection (5-6) and the dispatch (7)
- * separately.  stage_events is a HOST array of four cudaEvent_t handles (entries may be NULL),
- * recorded on cuda_stream: [0] before the first kernel, [1] after the contraction + score
- * epilogue, [2] after the selection, load update and combine weights, [3] after the dispatch.
+ * time the router + selection kernel (stages 1-6) and the dispatch kernels (7) separately.
+ * stage_events is a HOST array of four cudaEvent_t handles (entries may be NULL),
+ * recorded on cuda_stream: [0] before the first kernel, [1] and [2] after the kernel that
+ * runs the contraction, the score epilogue and the ordered selection with its load update,
+ * [3] after the dispatch kernels (which also write the combine weights).
  * With more than 64 layers the stages run once per group of 64 and the events keep the last
  * group's marks.  stage_events == NULL makes this identical to laser_route_layers.
  */

@@ -1,0 +1,53 @@
+// One launch for the router and the ordered selection.  The first n_layers blocks take the
+// selection role (one per layer); every other block routes one tile of router_rows tokens of
+// one layer and then publishes a ready flag for it.  Router blocks are numbered token-major
+// (the layer index varies fastest), so all layers advance together and each selection block
+// trails the router by about one tile instead of starting after the last router block.
+// Router blocks never wait, and there are far fewer selection blocks than the GPU can hold,
+// so the waits of the selection role always end; they are bounded all the same.
+#pragma once
+#include "k1_router.cuh"
+#include "k2_select.cuh"
+
+namespace laser {
+
+constexpr int kRouterWarps = kK2Threads / 32;
+
+template <int NT, int MT>
+__host__ __device__ constexpr int router_rows() { return kRouterWarps * MT * 16; }
+
+template <int NT, int MT>
+__host__ __device__ constexpr size_t router_smem_bytes() {
+  return sizeof(float) * kRouterWarps * MT * 16 * (NT * 8 + 1);
+}
+
+template <int NT, int MT, int KU>
+__global__ void __launch_bounds__(kK2Threads) k12_route_select(const RouteArgs A, int n_layers) {
+  extern __shared__ __align__(16) unsigned char dyn_smem[];
+  constexpr int RR = router_rows<NT, MT>();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if ((int)blockIdx.x < n_layers) {
+    const int layer = A.layer0 + blockIdx.x;
+    const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
+    k2_block(A, layer, dyn_smem, ready, RR);
+    return;
+  }
+  const int b = blockIdx.x - n_layers;
+  const int local_layer = b % n_layers;
+  const int rt = b / n_layers;
+  const long long tok0 = (long long)rt * RR + (long long)warp * (MT * 16);
+  if (tok0 < A.T) {
+    float* tile = reinterpret_cast<float*>(dyn_smem) + (size_t)warp * (MT * 16) * (NT * 8 + 1);
+    router_warp<NT, MT, KU>(A, local_layer, tok0, tile, lane);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
+                                        A.lay.ready);
+    __threadfence();
+    st_release(ready + rt, 1);
+  }
+}
+
+}  // namespace laser

@@ -85,21 +85,18 @@ __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int 
   }
 }
 
+// One warp routes ROWS = MT*16 consecutive tokens [tok0, tok0 + ROWS) of one layer.
 // NT: 8-expert column tiles (E padded up to NT*8).  MT: 16-row tiles per warp.
 // KU: chunks of 32 hidden elements issued per loop trip.
+// tile: this warp's shared-memory scratch of ROWS * (NT*8 + 1) floats.
 template <int NT, int MT, int KU>
-__global__ void __launch_bounds__(128) k1_router_mma(const RouteArgs A) {
-  extern __shared__ float smem_tile[];
+__device__ __forceinline__ void router_warp(const RouteArgs& A, int layer, long long tok0,
+                                            float* tile, int lane) {
   constexpr int ROWS = MT * 16;
   constexpr int EP = NT * 8;
   constexpr int LDS = EP + 1;
-
-  const int layer = blockIdx.y;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, q = lane & 3;
   const int T = A.T, d = A.d, E = A.E;
-  const long long tok0 = A.tok_begin + ((long long)blockIdx.x * 4 + warp) * ROWS;
-  if (tok0 >= A.tok_end) return;
 
   const uint16_t* hid = A.hidden + (size_t)(A.layer0 + layer) * A.hidden_ls;
   const uint16_t* wg = A.wg + (size_t)(A.layer0 + layer) * A.wg_ls;
@@ -179,7 +176,6 @@ __global__ void __launch_bounds__(128) k1_router_mma(const RouteArgs A) {
   }
 
   // accumulators (+ bias) -> this warp's shared-memory tile [ROWS][LDS]
-  float* tile = smem_tile + (size_t)warp * ROWS * LDS;
   const float* bias = A.bias ? A.bias + (size_t)(A.layer0 + layer) * E : nullptr;
 #pragma unroll
   for (int n = 0; n < NT; ++n) {
@@ -204,7 +200,7 @@ __global__ void __launch_bounds__(128) k1_router_mma(const RouteArgs A) {
   }
   __syncwarp();
 
-  const int rows_here = (int)min((long long)ROWS, (long long)A.tok_end - tok0);
+  const int rows_here = (int)min((long long)ROWS, (long long)T - tok0);
   if (A.logits_out) {
     float* out = A.logits_out + ((size_t)(A.layer0 + layer) * T + tok0) * E;
     for (int idx = lane; idx < rows_here * E; idx += 32) {

@@ -3,11 +3,7 @@
 // buffer entry point), no state between calls.
 #include "../../include/laser.h"
 
-#include <cstdlib>
-#include <mutex>
-
-#include "k1_router.cuh"
-#include "k2_select.cuh"
+#include "k12_fused.cuh"
 #include "k3_dispatch.cuh"
 
 using namespace laser;
@@ -34,78 +30,29 @@ int validate_params(const laser_params* p) {
 }
 
 template <int NT, int MT, int KU>
-cudaError_t launch_k1(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  constexpr int rows_per_block = 4 * MT * 16;
-  const size_t smem = sizeof(float) * 4 * MT * 16 * (NT * 8 + 1);
+cudaError_t launch_k12(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  size_t smem = router_smem_bytes<NT, MT>();
+  const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
+  if (smem2 > smem) smem = smem2;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k1_router_mma<NT, MT, KU>,
+    cudaError_t e = cudaFuncSetAttribute(k12_route_select<NT, MT, KU>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  const int ntok = a.tok_end - a.tok_begin;
-  dim3 grid((unsigned)((ntok + rows_per_block - 1) / rows_per_block), (unsigned)n_layers);
-  k1_router_mma<NT, MT, KU><<<grid, 128, smem, s>>>(a);
+  constexpr int RR = router_rows<NT, MT>();
+  const unsigned router_tiles = (unsigned)((a.T + RR - 1) / RR);
+  k12_route_select<NT, MT, KU><<<n_layers * (1 + router_tiles), kK2Threads, smem, s>>>(a, n_layers);
   return cudaGetLastError();
 }
 
-cudaError_t launch_k1_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
+cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
-  if (E <= 8) return launch_k1<1, 2, 4>(a, n_layers, s);
-  if (E <= 16) return launch_k1<2, 2, 4>(a, n_layers, s);
-  if (E <= 32) return launch_k1<4, 2, 2>(a, n_layers, s);
-  if (E <= 64) return launch_k1<8, 2, 2>(a, n_layers, s);
-  if (E <= 128) return launch_k1<16, 1, 2>(a, n_layers, s);
-  return launch_k1<32, 1, 1>(a, n_layers, s);
-}
-
-size_t k2_smem_bytes(int E, int c, int k) {
-  const size_t base = align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c);
-  if (c > 32 || k > 32) return base;  // wide fallback: no staged tiles
-  return base + 2 * k2_buffer_bytes(E, c);
-}
-
-// Per-device helper objects for overlapping the ordered selection of one token chunk with
-// the router kernel of the next: one high-priority side stream and a few events, created on
-// first use and kept until the process exits.
-constexpr int kMaxChunks = 16;
-struct DeviceAux {
-  bool ready = false;
-  cudaStream_t side = nullptr;
-  cudaEvent_t k1_done[kMaxChunks] = {};
-  cudaEvent_t side_done = nullptr;
-};
-DeviceAux g_aux[64];
-std::mutex g_aux_mutex;
-
-DeviceAux* get_aux() {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  DeviceAux& a = g_aux[dev];
-  if (!a.ready) {
-    int lo = 0, hi = 0;
-    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
-    if (cudaStreamCreateWithPriority(&a.side, cudaStreamNonBlocking, hi) != cudaSuccess)
-      return nullptr;
-    for (int i = 0; i < kMaxChunks; ++i)
-      if (cudaEventCreateWithFlags(&a.k1_done[i], cudaEventDisableTiming) != cudaSuccess)
-        return nullptr;
-    if (cudaEventCreateWithFlags(&a.side_done, cudaEventDisableTiming) != cudaSuccess)
-      return nullptr;
-    a.ready = true;
-  }
-  return &a;
-}
-
-// Tokens per chunk of the router/selection pipeline (multiple of the selection tile).
-int chunk_tokens(int T) {
-  static const int env = [] {
-    const char* v = std::getenv("LASER_CHUNK_TOKENS");
-    return v ? std::atoi(v) : 0;
-  }();
-  int ct = env > 0 ? env : 4096;
-  ct = ((ct + kK2MaxTile - 1) / kK2MaxTile) * kK2MaxTile;
-  while ((T + ct - 1) / ct > kMaxChunks) ct *= 2;
-  return ct;
+  if (E <= 8) return launch_k12<1, 2, 4>(a, n_layers, s);
+  if (E <= 16) return launch_k12<2, 2, 4>(a, n_layers, s);
+  if (E <= 32) return launch_k12<4, 2, 2>(a, n_layers, s);
+  if (E <= 64) return launch_k12<8, 2, 2>(a, n_layers, s);
+  if (E <= 128) return launch_k12<16, 1, 2>(a, n_layers, s);
+  return launch_k12<32, 1, 1>(a, n_layers, s);
 }
 
 // Enqueues all stages for layers [layer0, layer0 + n) of a batched call.
@@ -119,45 +66,19 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
     a.eps_high[l] = eps ? eps[layer0 + l] : p->eps_high;
     a.t_fix[l] = tfix ? tfix[layer0 + l] : p->t_fix;
   }
-  cudaError_t e = cudaSuccess;
   if (!mark(0)) return LASER_ERR_CUDA;
   if (a.T > 0) {
-    const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
-    if (smem2 > 48 * 1024) {
-      e = cudaFuncSetAttribute(k2_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
-      if (e != cudaSuccess) return LASER_ERR_CUDA;
-    }
-    const int ct = chunk_tokens(a.T);
-    const int n_chunks = (a.T + ct - 1) / ct;
-    if (n_chunks == 1) {
-      a.tok_begin = 0; a.tok_end = a.T;
-      if (launch_k1_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
-      if (!mark(1)) return LASER_ERR_CUDA;
-      k2_select<<<n, kK2Threads, smem2, s>>>(a);
-      if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-    } else {
-      // router kernel of chunk i+1 on the caller's stream overlaps the selection of chunk i
-      // on the side stream; the selection kernels run in chunk order and carry the loads
-      std::lock_guard<std::mutex> lock(g_aux_mutex);
-      DeviceAux* aux = get_aux();
-      if (!aux) return LASER_ERR_CUDA;
-      for (int ch = 0; ch < n_chunks; ++ch) {
-        a.tok_begin = ch * ct;
-        a.tok_end = a.tok_begin + ct < a.T ? a.tok_begin + ct : a.T;
-        if (launch_k1_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
-        if (cudaEventRecord(aux->k1_done[ch], s) != cudaSuccess) return LASER_ERR_CUDA;
-        if (cudaStreamWaitEvent(aux->side, aux->k1_done[ch], 0) != cudaSuccess)
-          return LASER_ERR_CUDA;
-        k2_select<<<n, kK2Threads, smem2, aux->side>>>(a);
-        if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-      }
-      if (!mark(1)) return LASER_ERR_CUDA;
-      if (cudaEventRecord(aux->side_done, aux->side) != cudaSuccess) return LASER_ERR_CUDA;
-      if (cudaStreamWaitEvent(s, aux->side_done, 0) != cudaSuccess) return LASER_ERR_CUDA;
-    }
-  } else if (!mark(1)) {
-    return LASER_ERR_CUDA;
+    // clear the router's ready flags of these layers (one strided memset), then one launch
+    // for the router and the ordered selection
+    const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 127) / 128 + 1);
+    if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
+                          (size_t)n, s) != cudaSuccess)
+      return LASER_ERR_CUDA;
+    a.tok_begin = 0;
+    a.tok_end = a.T;
+    if (launch_k12_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
   }
+  if (!mark(1)) return LASER_ERR_CUDA;
   if (!mark(2)) return LASER_ERR_CUDA;
   const size_t smem3 = sizeof(int32_t) * kK3Warps * a.E;
   dim3 g3((unsigned)a.lay.n_blk, (unsigned)n);

@@ -16,6 +16,7 @@ struct WorkspaceLayout {
   size_t sel_rank;     // uint8  [T, k]     rank positions chosen by the load-aware scan
   size_t pair_dst;     // int32  [T*k]      destination index in perm of pair t*k+j (score order)
   size_t blk_hist;     // int32  [n_blk, E] dispatch block histograms, then block bases
+  size_t ready;        // int32  [ceil(T/128)] router tiles published to the selection role
   size_t total;        // bytes per layer, multiple of 256
   int n_blk;           // dispatch blocks per layer
 };
@@ -36,6 +37,7 @@ inline WorkspaceLayout make_layout(int T, int E, int k, int c) {
   w.n_blk = (int)((pairs + kDispatchPairsPerBlock - 1) / kDispatchPairsPerBlock);
   if (w.n_blk < 1) w.n_blk = 1;
   w.blk_hist = off;     off = align256(off + sizeof(int32_t) * (size_t)w.n_blk * E);
+  w.ready = off;        off = align256(off + sizeof(int32_t) * (size_t)((T + 127) / 128 + 1));
   w.total = off;
   return w;
 }
