@@ -41,7 +41,9 @@ enum {
   LASER_ERR_UNSUPPORTED = -2,      /* a documented but unimplemented mode */
   LASER_ERR_WORKSPACE_TOO_SMALL = -3,
   LASER_ERR_MISALIGNED = -4,       /* hidden / W_g base or row stride not 16-byte aligned */
-  LASER_ERR_CUDA = -5              /* a CUDA runtime call failed (launch error) */
+  LASER_ERR_CUDA = -5,             /* a CUDA runtime call failed (launch error) */
+  LASER_ERR_STATIC_SCRATCH = -6    /* laser_route_static: the parameters need more scratch than
+                                      LASER_STATIC_SCRATCH_BYTES */
 };
 
 /* Bits in *status_word.
@@ -188,6 +190,43 @@ int laser_route_host(int32_t n_layers,
                      int32_t* expert_ids, float* weights, int32_t* offsets, int32_t* perm,
                      int32_t* status_out,
                      void* arena, size_t arena_bytes, void* cuda_stream);
+
+/* Size of the scratch array built into the library for laser_route_static (4 MiB). */
+enum { LASER_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 };
+
+/*
+ * laser_route for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of the library, not a step of the method.)
+ *
+ * laser_route needs a scratch buffer that its caller allocates.  Some callers have no way to
+ * do that: code that runs inside another program's fixed memory pool, a service whose
+ * allocator is frozen once it has started, a routine that may not call cudaMalloc because an
+ * allocation would stall every stream of the process.  This entry point takes the same
+ * inputs and outputs as laser_route, with the same results, but its scratch is an array of
+ * LASER_STATIC_SCRATCH_BYTES bytes that is part of the library itself.  The cost: every GPU
+ * on which the library is loaded gives up that much memory until the process exits.
+ *
+ *   - The call itself allocates and frees nothing, on the host side of CUDA or the device.
+ *   - Parameters whose laser_workspace_bytes() is larger than LASER_STATIC_SCRATCH_BYTES are
+ *     refused with LASER_ERR_STATIC_SCRATCH and nothing is launched.  One layer of 16384
+ *     tokens with k = 6, c = 8 needs about 1.2 MiB.
+ *   - The device that owns cuda_stream must be the current device.
+ *   - The first call on each device looks up the array's device address (a runtime query,
+ *     once per device, cached under a lock).  Make that first call outside any stream
+ *     capture.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call
+ *     left; the call clears the part that has to start at zero on the stream.  Two calls
+ *     whose kernels can overlap on the GPU (different streams without an ordering between
+ *     them) race on the array and give undefined results: order them.
+ *
+ * Arguments, return value and status_word are those of laser_route, without workspace and
+ * workspace_bytes.
+ */
+int laser_route_static(const void* hidden, const void* w_g, const float* bias,
+                       int32_t* loads, const int32_t* expert_to_bin, int32_t* bin_loads,
+                       const laser_params* p,
+                       int32_t* expert_ids, float* weights, int32_t* offsets, int32_t* perm,
+                       float* logits_out, int32_t* status_word, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -109,6 +109,8 @@ extern "C" const char* laser_strerror(int status) {
     case LASER_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case LASER_ERR_MISALIGNED: return "pointer or row stride not 16-byte aligned";
     case LASER_ERR_CUDA: return "CUDA runtime error";
+    case LASER_ERR_STATIC_SCRATCH:
+      return "parameters need more scratch than the library's built-in array holds";
     default: return "unknown status";
   }
 }

@@ -27,12 +27,14 @@ ERR_UNSUPPORTED = -2
 ERR_WORKSPACE_TOO_SMALL = -3
 ERR_MISALIGNED = -4
 ERR_CUDA = -5
+ERR_STATIC_SCRATCH = -6
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 DEV_LOAD_OVERFLOW = 1
 MAX_EXPERTS = 256
 
 EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_route",
            "laser_route_layers", "laser_route_layers_profiled", "laser_host_arena_bytes",
-           "laser_route_host")
+           "laser_route_host", "laser_route_static")
 
 
 class LaserParams(ctypes.Structure):
@@ -65,6 +67,9 @@ _lib.laser_host_arena_bytes.restype = ctypes.c_int
 _lib.laser_route_host.argtypes = [_i32, _vp, _vp, _vp, _vp, _vp, _vp, _pp, _vp, _vp,
                                   _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.laser_route_host.restype = ctypes.c_int
+_lib.laser_route_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _pp, _vp, _vp, _vp, _vp, _vp,
+                                    _vp, _vp]
+_lib.laser_route_static.restype = ctypes.c_int
 
 
 class LaserError(RuntimeError):
@@ -187,6 +192,26 @@ def route(hidden, w_g, bias, loads, p: LaserParams, *, bin_loads=None, **kw) -> 
                      p, bin_loads=None if bin_loads is None else bin_loads[None], **kw)
     return RouteResult(r.expert_ids[0], r.weights[0], r.offsets[0], r.perm[0], loads, bin_loads,
                        None if r.logits is None else r.logits[0], r.status)
+
+
+def route_static(hidden, w_g, bias, loads, p: LaserParams, out: RouteResult, *,
+                 expert_to_bin=None, bin_loads=None, stream=None) -> RouteResult:
+    """laser_route_static for one layer, for callers that must not allocate: every tensor,
+    the outputs in ``out`` included, is preallocated by the caller (hidden [T,d], w_g [E,d],
+    bias [E] or None, loads [E] in place, out.expert_ids / weights [T,k], out.offsets [E+1],
+    out.perm [T*k], out.logits [T,E] or None, out.status [1]); the scratch is the library's
+    built-in array, so no workspace is passed.  Raises LaserError(ERR_STATIC_SCRATCH) when
+    the shape needs more than STATIC_SCRATCH_BYTES."""
+    import torch
+
+    s = torch.cuda.current_stream(hidden.device) if stream is None else stream
+    rc = _lib.laser_route_static(
+        _ptr(hidden), _ptr(w_g), _ptr(bias), _ptr(loads), _ptr(expert_to_bin), _ptr(bin_loads),
+        ctypes.byref(p), _ptr(out.expert_ids), _ptr(out.weights), _ptr(out.offsets),
+        _ptr(out.perm), _ptr(out.logits), _ptr(out.status), s.cuda_stream)
+    if rc != OK:
+        raise LaserError(rc)
+    return out
 
 
 def route_host(hidden, w_g, bias, loads, p: LaserParams, arena, *, expert_to_bin=None,
