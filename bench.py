@@ -318,11 +318,25 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-layers", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eps-high", type=float, default=None,
+                    help="override eps_high of every layer (0 = vanilla top-k, 2 = always expand)")
+    ap.add_argument("--t-fix", type=float, default=None, help="override t_fix of every layer")
+    ap.add_argument("--c", type=int, default=None, help="override the trimming size c")
     args = ap.parse_args()
 
     from paper_2510_03293_b200 import synth
 
     w = synth.WORKLOADS[args.workload]
+    over = {}
+    if args.eps_high is not None:
+        over["eps_high"] = (args.eps_high,)
+    if args.t_fix is not None:
+        over["t_fix"] = args.t_fix
+    if args.c is not None:
+        over["c"] = args.c
+    if over:
+        import dataclasses
+        w = dataclasses.replace(w, **over)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -16,30 +16,38 @@ constexpr int kRouterWarps = kK2Threads / 32;
 template <int NT, int MT>
 __host__ __device__ constexpr int router_rows() { return kRouterWarps * MT * 16; }
 
-template <int NT, int MT>
-__host__ __device__ constexpr size_t router_smem_bytes() {
+// logits tile of the block
+__host__ __device__ inline size_t router_smem_bytes(int NT, int MT) {
   return sizeof(float) * kRouterWarps * MT * 16 * (NT * 8 + 1);
 }
 
-template <int NT, int MT, int KU>
+template <int NT, int MT, int KU, int CMAX>
 __global__ void __launch_bounds__(kK2Threads) k12_route_select(const RouteArgs A, int n_layers) {
-  extern __shared__ __align__(16) unsigned char dyn_smem[];
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
   constexpr int RR = router_rows<NT, MT>();
+  constexpr int LDS = NT * 8 + 1;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if ((int)blockIdx.x < n_layers) {
     const int layer = A.layer0 + blockIdx.x;
     const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
-    k2_block(A, layer, dyn_smem, ready, RR);
+    k2_block<CMAX, (NT * 8 <= 32)>(A, layer, dyn_smem, ready, RR);
     return;
   }
   const int b = blockIdx.x - n_layers;
   const int local_layer = b % n_layers;
   const int rt = b / n_layers;
+  float* tiles = reinterpret_cast<float*>(dyn_smem);
   const long long tok0 = (long long)rt * RR + (long long)warp * (MT * 16);
-  if (tok0 < A.T) {
-    float* tile = reinterpret_cast<float*>(dyn_smem) + (size_t)warp * (MT * 16) * (NT * 8 + 1);
-    router_warp<NT, MT, KU>(A, local_layer, tok0, tile, lane);
+  if (tok0 < A.T) router_warp<NT, MT, KU>(A, local_layer, tok0, tiles + (size_t)warp * (MT * 16) * LDS, lane);
+  if (MT == 2) {
+    // a warp's 32 rows are one group: no block-wide hand-over needed
+    if (tok0 < A.T) group_epilogue(A, local_layer, tok0, tiles + (size_t)warp * 32 * LDS, LDS, lane);
+  } else {
+    __syncthreads();
+    const long long gtok0 = (long long)rt * RR + (long long)warp * 32;
+    if (warp * 32 < RR && gtok0 < A.T)
+      group_epilogue(A, local_layer, gtok0, tiles + (size_t)warp * 32 * LDS, LDS, lane);
   }
   __syncthreads();
   if (tid == 0) {

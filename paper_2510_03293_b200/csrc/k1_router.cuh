@@ -85,7 +85,8 @@ __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int 
   }
 }
 
-// One warp routes ROWS = MT*16 consecutive tokens [tok0, tok0 + ROWS) of one layer.
+// One warp contracts ROWS = MT*16 consecutive tokens [tok0, tok0 + ROWS) of one layer with W_g
+// and leaves their fp32 logits (+ bias) in its shared-memory tile.
 // NT: 8-expert column tiles (E padded up to NT*8).  MT: 16-row tiles per warp.
 // KU: chunks of 32 hidden elements issued per loop trip.
 // tile: this warp's shared-memory scratch of ROWS * (NT*8 + 1) floats.
@@ -209,17 +210,22 @@ __device__ __forceinline__ void router_warp(const RouteArgs& A, int layer, long 
     }
   }
 
+}
+
+// Score epilogue of up to 32 tokens [tok0, tok0 + 32) by one warp, lane = token.  rows: the
+// tokens' logits in shared memory, row stride lds floats.
+__device__ __forceinline__ void group_epilogue(const RouteArgs& A, int layer, long long tok0,
+                                               const float* rows, int lds, int lane) {
+  const long long t = tok0 + lane;
+  if (t >= A.T) return;
   unsigned char* ws = A.ws + (size_t)(A.layer0 + layer) * A.ws_ls;
   const int k = A.k, c = A.c;
-  for (int r = lane; r < rows_here; r += 32) {
-    const long long t = tok0 + r;
-    const size_t lt = (size_t)(A.layer0 + layer) * T + t;
-    token_epilogue(tile + r * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
-                   reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
-                   ws + A.lay.cand_ids + (size_t)t * c,
-                   reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
-                   A.expert_ids + lt * k, A.weights + lt * k);
-  }
+  const size_t lt = (size_t)(A.layer0 + layer) * A.T + t;
+  token_epilogue(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
+                 reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
+                 ws + A.lay.cand_ids + (size_t)t * c,
+                 reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
+                 A.expert_ids + lt * k, A.weights + lt * k);
 }
 
 }  // namespace laser

@@ -29,30 +29,41 @@ int validate_params(const laser_params* p) {
   return LASER_OK;
 }
 
-template <int NT, int MT, int KU>
+template <int NT, int MT, int KU, int CMAX>
 cudaError_t launch_k12(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  size_t smem = router_smem_bytes<NT, MT>();
+  size_t smem = router_smem_bytes(NT, MT);
   const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
   if (smem2 > smem) smem = smem2;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k12_route_select<NT, MT, KU>,
+    cudaError_t e = cudaFuncSetAttribute(k12_route_select<NT, MT, KU, CMAX>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   constexpr int RR = router_rows<NT, MT>();
   const unsigned router_tiles = (unsigned)((a.T + RR - 1) / RR);
-  k12_route_select<NT, MT, KU><<<n_layers * (1 + router_tiles), kK2Threads, smem, s>>>(a, n_layers);
+  k12_route_select<NT, MT, KU, CMAX>
+      <<<n_layers * (1 + router_tiles), kK2Threads, smem, s>>>(a, n_layers);
   return cudaGetLastError();
+}
+
+// The selection sorts CMAX >= c candidate keys in registers; pick the smallest network.
+template <int NT, int MT, int KU>
+cudaError_t launch_k12_for_c(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  constexpr int EP = NT * 8;
+  if (EP >= 4 && a.c <= 4) return launch_k12<NT, MT, KU, 4>(a, n_layers, s);
+  if (EP >= 8 && a.c <= 8) return launch_k12<NT, MT, KU, 8>(a, n_layers, s);
+  if (EP >= 16 && a.c <= 16) return launch_k12<NT, MT, KU, (EP >= 16 ? 16 : 8)>(a, n_layers, s);
+  return launch_k12<NT, MT, KU, (EP >= 32 ? 32 : EP)>(a, n_layers, s);
 }
 
 cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
-  if (E <= 8) return launch_k12<1, 2, 4>(a, n_layers, s);
-  if (E <= 16) return launch_k12<2, 2, 4>(a, n_layers, s);
-  if (E <= 32) return launch_k12<4, 2, 2>(a, n_layers, s);
-  if (E <= 64) return launch_k12<8, 2, 2>(a, n_layers, s);
-  if (E <= 128) return launch_k12<16, 1, 2>(a, n_layers, s);
-  return launch_k12<32, 1, 1>(a, n_layers, s);
+  if (E <= 8) return launch_k12_for_c<1, 1, 8>(a, n_layers, s);
+  if (E <= 16) return launch_k12_for_c<2, 2, 4>(a, n_layers, s);
+  if (E <= 32) return launch_k12_for_c<4, 2, 2>(a, n_layers, s);
+  if (E <= 64) return launch_k12_for_c<8, 2, 2>(a, n_layers, s);
+  if (E <= 128) return launch_k12_for_c<16, 1, 2>(a, n_layers, s);
+  return launch_k12_for_c<32, 1, 1>(a, n_layers, s);
 }
 
 // Enqueues all stages for layers [layer0, layer0 + n) of a batched call.
@@ -67,32 +78,31 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
     a.t_fix[l] = tfix ? tfix[layer0 + l] : p->t_fix;
   }
   if (!mark(0)) return LASER_ERR_CUDA;
-  if (a.T > 0) {
-    // clear the router's ready flags of these layers (one strided memset), then one launch
-    // for the router and the ordered selection
-    const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 127) / 128 + 1);
-    if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
-                          (size_t)n, s) != cudaSuccess)
+  if (a.T == 0) {
+    // nothing to route: the call's offsets are all zero, loads and bins stay as they are
+    if (cudaMemsetAsync(a.offsets + (size_t)layer0 * (a.E + 1), 0,
+                        sizeof(int32_t) * (size_t)n * (a.E + 1), s) != cudaSuccess)
       return LASER_ERR_CUDA;
-    a.tok_begin = 0;
-    a.tok_end = a.T;
-    if (launch_k12_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
+    return (mark(1) && mark(2) && mark(3)) ? LASER_OK : LASER_ERR_CUDA;
   }
+  // clear the router's ready flags of these layers (one strided memset), then one launch for
+  // the router and the ordered selection, one for the dispatch
+  const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 127) / 128 + 1);
+  if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
+                        (size_t)n, s) != cudaSuccess)
+    return LASER_ERR_CUDA;
+  if (launch_k12_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
   if (!mark(1)) return LASER_ERR_CUDA;
   if (!mark(2)) return LASER_ERR_CUDA;
-  const size_t smem3 = sizeof(int32_t) * kK3Warps * a.E;
-  dim3 g3((unsigned)a.lay.n_blk, (unsigned)n);
-  k3_hist<<<g3, kK3Threads, smem3, s>>>(a);
+  const int warps = k3_warps_per_block(a.E, a.k);
+  const size_t smem3 = (size_t)warps * k3_warp_smem_bytes(a.E, a.k);
+  if (smem3 > 48 * 1024 &&
+      cudaFuncSetAttribute(k3_dispatch, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem3) != cudaSuccess)
+    return LASER_ERR_CUDA;
+  dim3 g3((unsigned)((a.lay.n_groups + warps - 1) / warps), (unsigned)n);
+  k3_dispatch<<<g3, warps * 32, smem3, s>>>(a);
   if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-  k3_scan<<<n, kK3Threads, 0, s>>>(a);
-  if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-  k3_rank<<<g3, kK3Threads, smem3, s>>>(a);
-  if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-  if (a.T > 0) {
-    dim3 gf((unsigned)((a.T + 127) / 128), (unsigned)n);
-    k3_finalize<<<gf, 128, 0, s>>>(a);
-    if (cudaGetLastError() != cudaSuccess) return LASER_ERR_CUDA;
-  }
   if (!mark(3)) return LASER_ERR_CUDA;
   return LASER_OK;
 }

@@ -14,29 +14,25 @@ struct WorkspaceLayout {
   size_t cand_ids;     // uint8  [T, c]     ranking pi(0..c-1)
   size_t cand_scores;  // float  [T, c]     s_pi(j)
   size_t sel_rank;     // uint8  [T, k]     rank positions chosen by the load-aware scan
-  size_t pair_dst;     // int32  [T*k]      destination index in perm of pair t*k+j (score order)
-  size_t blk_hist;     // int32  [n_blk, E] dispatch block histograms, then block bases
-  size_t ready;        // int32  [ceil(T/128)] router tiles published to the selection role
+  size_t grp_base;     // int32  [n_groups, E]  per-expert count of this call's assignments made
+                       //                   before the group (load at group start minus L_in)
+  size_t ready;        // int32  [ceil(T/128)+1] router tiles published to the selection role
   size_t total;        // bytes per layer, multiple of 256
-  int n_blk;           // dispatch blocks per layer
+  int n_groups;        // ceil(T / 32): the ordered selection and the dispatch work on groups
+                       // of 32 consecutive tokens
 };
-
-constexpr int kDispatchPairsPerBlock = 4096;
 
 __host__ __device__ inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 inline WorkspaceLayout make_layout(int T, int E, int k, int c) {
   WorkspaceLayout w;
   size_t off = 0;
+  w.n_groups = (T + 31) / 32;
   w.cstar = off;        off = align256(off + sizeof(uint16_t) * (size_t)T);
   w.cand_ids = off;     off = align256(off + (size_t)T * c);
   w.cand_scores = off;  off = align256(off + sizeof(float) * (size_t)T * c);
   w.sel_rank = off;     off = align256(off + (size_t)T * k);
-  w.pair_dst = off;     off = align256(off + sizeof(int32_t) * (size_t)T * k);
-  long long pairs = (long long)T * k;
-  w.n_blk = (int)((pairs + kDispatchPairsPerBlock - 1) / kDispatchPairsPerBlock);
-  if (w.n_blk < 1) w.n_blk = 1;
-  w.blk_hist = off;     off = align256(off + sizeof(int32_t) * (size_t)w.n_blk * E);
+  w.grp_base = off;     off = align256(off + sizeof(int32_t) * (size_t)w.n_groups * E);
   w.ready = off;        off = align256(off + sizeof(int32_t) * (size_t)((T + 127) / 128 + 1));
   w.total = off;
   return w;
@@ -61,7 +57,6 @@ struct RouteArgs {
   int T, d, E, k, c, n_bins, renorm;
   long long ld_h, ld_w;
   int layer0;              // first layer of this launch
-  int tok_begin, tok_end;  // token range of this launch (router and selection kernels)
   float eps_high[kMaxLayersPerLaunch];
   float t_fix[kMaxLayersPerLaunch];
 };
