@@ -8,6 +8,7 @@
 #pragma once
 #include "k1_router.cuh"
 #include "k2_select.cuh"
+#include "k1_router_tc.cuh"
 
 namespace laser {
 
@@ -51,6 +52,32 @@ __global__ void __launch_bounds__(kK2Threads) k12_route_select(const RouteArgs A
   }
   __syncthreads();
   if (tid == 0) {
+    int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
+                                        A.lay.ready);
+    __threadfence();
+    st_release(ready + rt, 1);
+  }
+}
+
+// The same launch shape with the tensor-memory router (E > 32): the first n_layers blocks
+// select, every other block routes one tile of 128 tokens.
+template <int N, int CMAX>
+__global__ void __launch_bounds__(kK2Threads, tc_min_blocks<N>())
+k12_route_select_tc(const RouteArgs A, int n_layers, const __grid_constant__ CUtensorMap map_h,
+                    const __grid_constant__ CUtensorMap map_w) {
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
+  if ((int)blockIdx.x < n_layers) {
+    const int layer = A.layer0 + blockIdx.x;
+    const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
+    k2_block<CMAX, false>(A, layer, dyn_smem, ready, kTcTileM);
+    return;
+  }
+  const int b = blockIdx.x - n_layers;
+  const int local_layer = b % n_layers;
+  const int rt = b / n_layers;
+  router_tc_block<N>(A, &map_h, &map_w, local_layer, rt, dyn_smem);
+  // router_tc_block ends with a block barrier after the last record was written
+  if (threadIdx.x == 0) {
     int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
                                         A.lay.ready);
     __threadfence();

@@ -56,8 +56,83 @@ cudaError_t launch_k12_for_c(const RouteArgs& a, int n_layers, cudaStream_t s) {
   return launch_k12<NT, MT, KU, (EP >= 32 ? 32 : EP)>(a, n_layers, s);
 }
 
+// ---- tensor-memory router (E > 32): TMA tensor maps and launch --------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) !=
+            cudaSuccess || q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// 2-D bf16 view [rows, d] with row pitch ld elements; boxes of box_rows x 64 elements stored
+// with the 128-byte swizzle; out-of-range elements read as zero.
+bool make_map(CUtensorMap* m, const void* base, long long rows, int d, long long ld, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || rows <= 0 || rows > 0xffffffffLL) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kTcSliceK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int N, int CMAX>
+cudaError_t launch_k12_tc(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
+                          const CUtensorMap& mw, cudaStream_t s) {
+  size_t smem = tc_smem_bytes<N>();
+  const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
+  if (smem2 > smem) smem = smem2;
+  cudaError_t e = cudaFuncSetAttribute(k12_route_select_tc<N, CMAX>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const unsigned tiles = (unsigned)((a.T + kTcTileM - 1) / kTcTileM);
+  k12_route_select_tc<N, CMAX><<<n_layers * (1 + tiles), kK2Threads, smem, s>>>(a, n_layers, mh, mw);
+  return cudaGetLastError();
+}
+
+template <int N>
+cudaError_t launch_k12_tc_for_c(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
+                                const CUtensorMap& mw, cudaStream_t s) {
+  if (a.c <= 4) return launch_k12_tc<N, 4>(a, n_layers, mh, mw, s);
+  if (a.c <= 8) return launch_k12_tc<N, 8>(a, n_layers, mh, mw, s);
+  if (a.c <= 16) return launch_k12_tc<N, 16>(a, n_layers, mh, mw, s);
+  return launch_k12_tc<N, 32>(a, n_layers, mh, mw, s);
+}
+
+// Returns false if the tensor maps cannot be built for this call (the caller then uses the
+// warp-level router, which has no such requirement).
+bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, cudaError_t* err) {
+  // hidden and W_g of the layers of this launch as one [layers*T, d] / [layers*E, d] matrix
+  if (a.hidden_ls != (long long)a.T * a.ld_h || a.wg_ls != (long long)a.E * a.ld_w) return false;
+  const int N = a.E <= 64 ? 64 : (a.E <= 128 ? 128 : 256);
+  CUtensorMap mh, mw;
+  const long long total_layers = (long long)a.layer0 + n_layers;
+  if (!make_map(&mh, a.hidden, total_layers * a.T, a.d, a.ld_h, kTcTileM)) return false;
+  if (!make_map(&mw, a.wg, total_layers * a.E, a.d, a.ld_w, N)) return false;
+  if (N == 64) *err = launch_k12_tc_for_c<64>(a, n_layers, mh, mw, s);
+  else if (N == 128) *err = launch_k12_tc_for_c<128>(a, n_layers, mh, mw, s);
+  else *err = launch_k12_tc_for_c<256>(a, n_layers, mh, mw, s);
+  return true;
+}
+
 cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
+  if (E > 32) {
+    cudaError_t err = cudaSuccess;
+    if (launch_k12_tensor_memory(a, n_layers, s, &err)) return err;
+  }
   if (E <= 8) return launch_k12_for_c<1, 1, 8>(a, n_layers, s);
   if (E <= 16) return launch_k12_for_c<2, 2, 4>(a, n_layers, s);
   if (E <= 32) return launch_k12_for_c<4, 2, 2>(a, n_layers, s);
