@@ -187,3 +187,47 @@ def test_load_overflow_sets_the_status_bit(cuda_device):
     assert g["status"] & 1
     L1 = np.zeros(8, np.int32)
     assert run_gpu(cuda_device, hb, wb, bias, L1, 2, 4, 0.64, 0.6)["status"] == 0
+
+
+def _route_layers_strided(dev, hb, wb, bias, ld_h, ld_w, k, c, eps, tfix, B):
+    """Routes [L,T,d] inputs stored with row pitches ld_h / ld_w (> d, padded with NaN bits so
+    that any read of the padding shows up in the logits)."""
+    import torch
+
+    from paper_2510_03293_b200 import laser
+
+    L, T, d = hb.shape
+    E = wb.shape[1]
+    hp = np.full((L, T, ld_h), 0x7FC0, np.uint16); hp[:, :, :d] = hb
+    wp = np.full((L, E, ld_w), 0x7FC0, np.uint16); wp[:, :, :d] = wb
+    p = laser.make_params(T, d, E, k, c, eps, tfix, 1, B, ld_hidden=ld_h, ld_w=ld_w)
+    loads = torch.zeros((L, E), dtype=torch.int32, device=dev)
+    bins = torch.zeros((L, B), dtype=torch.int32, device=dev)
+    r = laser.route_layers(to_dev_bf16(hp, dev), to_dev_bf16(wp, dev),
+                           torch.from_numpy(bias).to(dev), loads, p, bin_loads=bins,
+                           want_logits=True)
+    torch.cuda.synchronize()
+    return r, loads, bins
+
+
+@pytest.mark.parametrize("L,T,d,E,k,c,ld_h,ld_w", [
+    (3, 200, 264, 64, 6, 8, 264, 264),      # tensor-memory router: tiles straddle layers, d % 64 != 0
+    (2, 333, 520, 100, 5, 12, 528, 536),    # ... with padded rows and 128 accumulator columns
+    (2, 150, 256, 256, 8, 16, 320, 256),    # ... 256 accumulator columns, two-pass epilogue
+    (3, 300, 264, 8, 2, 4, 272, 280),       # warp-level router with padded rows
+])
+def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, L, T, d, E, k, c, ld_h, ld_w):
+    layers = [layer(T, d, E, seed=200 + l + E, sigma=0.05) for l in range(L)]
+    hb = np.stack([x[0] for x in layers]); wb = np.stack([x[1] for x in layers])
+    bias = np.stack([x[2] for x in layers])
+    B = 4
+    r, loads, bins = _route_layers_strided(cuda_device, hb, wb, bias, ld_h, ld_w, k, c, 0.5, 0.5, B)
+    assert int(r.status.item()) == 0
+    for l in range(L):
+        g = dict(expert_ids=r.expert_ids[l].cpu().numpy(), weights=r.weights[l].cpu().numpy(),
+                 offsets=r.offsets[l].cpu().numpy(), perm=r.perm[l].cpu().numpy(),
+                 loads=loads[l].cpu().numpy(), bin_loads=bins[l].cpu().numpy(),
+                 logits=r.logits[l].cpu().numpy(), status=0)
+        assert np.isfinite(g["logits"]).all()
+        check_against_oracle(g, hb[l], wb[l], bias[l], np.zeros(E, np.int32), k, c, 0.5, 0.5, 1, B,
+                             bins0=np.zeros(B, np.int32))
