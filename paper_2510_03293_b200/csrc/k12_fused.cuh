@@ -59,6 +59,31 @@ __global__ void __launch_bounds__(kK2Threads) k12_route_select(const RouteArgs A
   }
 }
 
+// The same launch shape with the split-K router for calls with few tokens: every router block
+// routes 16 tokens.
+template <int NT, int KU, int CMAX>
+__global__ void __launch_bounds__(kK2Threads)
+k12_route_select_splitk(const RouteArgs A, int n_layers) {
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
+  if ((int)blockIdx.x < n_layers) {
+    const int layer = A.layer0 + blockIdx.x;
+    const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
+    k2_block<CMAX, (NT * 8 <= 32)>(A, layer, dyn_smem, ready, 16);
+    return;
+  }
+  const int b = blockIdx.x - n_layers;
+  const int local_layer = b % n_layers;
+  const int rt = b / n_layers;
+  router_splitk_block<NT, KU>(A, local_layer, rt, reinterpret_cast<float*>(dyn_smem));
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
+                                        A.lay.ready);
+    __threadfence();
+    st_release(ready + rt, 1);
+  }
+}
+
 // The same launch shape with the tensor-memory router (E > 32): the first n_layers blocks
 // select, every other block routes one tile of 128 tokens.
 template <int N, int CMAX>

@@ -85,6 +85,155 @@ __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int 
   }
 }
 
+// Score epilogue of 4 tokens by one warp, 8 lanes per token (same arithmetic, operation by
+// operation, as token_epilogue on a shared-memory row):
+//   ranking pi by (logit desc, index asc);  e_i = exp32(x_i - x_max);
+//   Z = eight interleaved running sums a_j = sum_{i = j mod 8, ascending} e_i combined as
+//       ((a0+a1)+(a2+a3))+((a4+a5)+(a6+a7));  s = e / Z;  M_k left to right;
+//   top-k branch iff M_k >= eps_high;  otherwise c* = max(k, #{j < c : s_pi(j) >= t_fix*s_pi(0)}).
+// row: the token's logits in shared memory (nullptr-safe only through write = false with a
+// valid row).  Lane j of the group owns experts 8m + j.  All 32 lanes must call.
+template <int N>
+__device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, int E, int k, int c,
+                                                      float eps_high, float t_fix, int renorm,
+                                                      bool write, uint16_t* cstar,
+                                                      uint8_t* cand_ids, float* cand_scores,
+                                                      int32_t* expert_ids, float* weights) {
+  constexpr int EPL = N / 8;
+  const float ninf = __int_as_float(0xff800000);
+  float x[EPL];
+  float xmax = ninf;
+#pragma unroll
+  for (int m = 0; m < EPL; ++m) {
+    const int i = 8 * m + j;
+    x[m] = i < E ? row[i] : ninf;
+    xmax = fmaxf(xmax, x[m]);
+  }
+#pragma unroll
+  for (int s = 1; s < 8; s <<= 1) xmax = fmaxf(xmax, __shfl_xor_sync(0xffffffffu, xmax, s));
+  float a = 0.0f;
+#pragma unroll
+  for (int m = 0; m < EPL; ++m)
+    if (8 * m + j < E) a = __fadd_rn(a, exp32(__fsub_rn(x[m], xmax)));
+  float Z = a;
+#pragma unroll
+  for (int s = 1; s < 8; s <<= 1) Z = __fadd_rn(Z, __shfl_xor_sync(0xffffffffu, Z, s));
+
+  float prev_x = __int_as_float(0x7f800000);  // +inf
+  int prev_i = -1;
+  if (c > 32) {
+    // wide candidate lists (rare): score every rank as it is found
+    float Mk = 0.0f, thr = 0.0f;
+    int mprime = 0;
+#pragma unroll 1
+    for (int r = 0; r < c; ++r) {
+      float bx = ninf;
+      int bi = 0x7fffffff;
+#pragma unroll
+      for (int m = 0; m < EPL; ++m) {
+        const int i = 8 * m + j;
+        const float xi = x[m];
+        const bool after_prev = (xi < prev_x) || (xi == prev_x && i > prev_i);
+        if (i < E && after_prev && xi > bx) { bx = xi; bi = i; }
+      }
+#pragma unroll
+      for (int s = 1; s < 8; s <<= 1) {
+        const float ox = __shfl_xor_sync(0xffffffffu, bx, s);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
+        if (ox > bx || (ox == bx && oi < bi)) { bx = ox; bi = oi; }
+      }
+      const float sr = __fdiv_rn(exp32(__fsub_rn(bx, xmax)), Z);
+      if (r == 0) { thr = __fmul_rn(t_fix, sr); Mk = sr; }
+      else if (r < k) Mk = __fadd_rn(Mk, sr);
+      if (sr >= thr) ++mprime;
+      if (write && j == 0) {
+        cand_ids[r] = (uint8_t)bi;
+        cand_scores[r] = sr;
+        if (r < k) { expert_ids[r] = bi; weights[r] = sr; }
+      }
+      prev_x = bx;
+      prev_i = bi;
+    }
+    if (!write || j != 0) return;
+    const bool top_k_branch = (Mk >= eps_high);
+    *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
+    if (top_k_branch && renorm)
+      for (int q = 0; q < k; ++q) weights[q] = __fdiv_rn(weights[q], Mk);
+    return;
+  }
+  // ranking: c rounds of "best remaining" (local scan, then a 3-step butterfly over the group);
+  // lane j keeps the results of ranks j, j+8, j+16, j+24
+  float kx[4] = {ninf, ninf, ninf, ninf};
+  int ki[4] = {0, 0, 0, 0};
+#pragma unroll 1
+  for (int r = 0; r < c; ++r) {
+    float bx = ninf;
+    int bi = 0x7fffffff;
+#pragma unroll
+    for (int m = 0; m < EPL; ++m) {
+      const int i = 8 * m + j;
+      const float xi = x[m];
+      const bool after_prev = (xi < prev_x) || (xi == prev_x && i > prev_i);
+      if (i < E && after_prev && xi > bx) { bx = xi; bi = i; }
+    }
+#pragma unroll
+    for (int s = 1; s < 8; s <<= 1) {
+      const float ox = __shfl_xor_sync(0xffffffffu, bx, s);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
+      if (ox > bx || (ox == bx && oi < bi)) { bx = ox; bi = oi; }
+    }
+    if ((r & 7) == j) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if ((r >> 3) == q) { kx[q] = bx; ki[q] = bi; }
+    }
+    prev_x = bx;
+    prev_i = bi;
+  }
+  // scores of this lane's ranks
+  float sc[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    sc[q] = (8 * q + j < c) ? __fdiv_rn(exp32(__fsub_rn(kx[q], xmax)), Z) : 0.0f;
+  // M_k = s_pi(0) + ... + s_pi(k-1), left to right; rank r lives in lane r % 8, slot r / 8
+  const int gbase = (threadIdx.x & 31) & ~7;
+  float Mk = 0.0f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (8 * q < k) {   // uniform over the warp
+#pragma unroll
+      for (int l = 0; l < 8; ++l) {
+        const float v = __shfl_sync(0xffffffffu, sc[q], gbase + l);
+        const int r = 8 * q + l;
+        if (r < k) Mk = r == 0 ? v : __fadd_rn(Mk, v);
+      }
+    }
+  }
+  const float s0 = __shfl_sync(0xffffffffu, sc[0], gbase);
+  const float thr = __fmul_rn(t_fix, s0);
+  int mprime = 0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    if (8 * q + j < c && sc[q] >= thr) ++mprime;
+#pragma unroll
+  for (int s = 1; s < 8; s <<= 1) mprime += __shfl_xor_sync(0xffffffffu, mprime, s);
+  if (!write) return;
+  const bool top_k_branch = (Mk >= eps_high);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = 8 * q + j;
+    if (r < c) {
+      cand_ids[r] = (uint8_t)ki[q];
+      cand_scores[r] = sc[q];
+      if (r < k) {
+        expert_ids[r] = ki[q];
+        weights[r] = (top_k_branch && renorm) ? __fdiv_rn(sc[q], Mk) : sc[q];
+      }
+    }
+  }
+  if (j == 0) *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
+}
+
 // One warp contracts ROWS = MT*16 consecutive tokens [tok0, tok0 + ROWS) of one layer with W_g
 // and leaves their fp32 logits (+ bias) in its shared-memory tile.
 // NT: 8-expert column tiles (E padded up to NT*8).  MT: 16-row tiles per warp.
@@ -226,6 +375,143 @@ __device__ __forceinline__ void group_epilogue(const RouteArgs& A, int layer, lo
                  ws + A.lay.cand_ids + (size_t)t * c,
                  reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
                  A.expert_ids + lt * k, A.weights + lt * k);
+}
+
+
+// Router for calls with few tokens: one block routes 16 tokens, its 8 warps each contract one
+// eighth of the hidden dimension (so that many SMs share the streaming of a small input),
+// the partial sums meet in shared memory in a fixed order, and warps 0..3 score 4 tokens each.
+// NT: 8-expert column tiles.  smem: router_splitk_smem_bytes(NT).
+__host__ __device__ inline size_t router_splitk_smem_bytes(int NT) {
+  return sizeof(float) * (8 * 16 * NT * 8 + 16 * (NT * 8 + 8));
+}
+
+template <int NT, int KU>
+__device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int layer, int rt,
+                                                    float* smem) {
+  constexpr int EP = NT * 8;
+  constexpr int LDS = EP + 8;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, q = lane & 3;
+  const int T = A.T, d = A.d, E = A.E;
+  const long long tok0 = (long long)rt * 16;
+  const int abs_layer = A.layer0 + layer;
+  const uint16_t* hid = A.hidden + (size_t)abs_layer * A.hidden_ls;
+  const uint16_t* wg = A.wg + (size_t)abs_layer * A.wg_ls;
+
+  const uint16_t* arow[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    long long r = tok0 + h * 8 + g;
+    if (r > T - 1) r = T - 1;  // rows past the end re-read the last row; results dropped
+    arow[h] = hid + r * A.ld_h + q * 8;
+  }
+  const uint16_t* brow[NT];
+  bool bval[NT];
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    const int e = n * 8 + g;
+    bval[n] = e < E;
+    brow[n] = wg + (long long)(bval[n] ? e : 0) * A.ld_w + q * 8;
+  }
+  float acc[NT][4];
+#pragma unroll
+  for (int n = 0; n < NT; ++n)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[n][i] = 0.0f;
+
+  // this warp's chunks of 32 hidden elements: [c_begin, c_end)
+  const int chunks = (d + 31) / 32;
+  const int per = (chunks + 7) / 8;
+  const int c_begin = min(chunks, warp * per), c_end = min(chunks, c_begin + per);
+  int kc = c_begin;
+  // all fragments of KU chunks are requested before the first MMA: with 16 tokens per block
+  // there are few warps per SM, so the loads of one warp must overlap each other
+  for (; kc + KU <= c_end && (kc + KU) * 32 <= d; kc += KU) {
+    uint4 av[KU][2];
+    uint4 bv[KU][NT];
+#pragma unroll
+    for (int u = 0; u < KU; ++u) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) av[u][h] = ldg_stream(arow[h] + (kc + u) * 32);
+#pragma unroll
+      for (int n = 0; n < NT; ++n)
+        bv[u][n] = bval[n] ? __ldg(reinterpret_cast<const uint4*>(brow[n] + (kc + u) * 32))
+                           : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < KU; ++u) {
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        mma_bf16_16816(acc[n], av[u][0].x, av[u][1].x, av[u][0].y, av[u][1].y, bv[u][n].x,
+                       bv[u][n].y);
+        mma_bf16_16816(acc[n], av[u][0].z, av[u][1].z, av[u][0].w, av[u][1].w, bv[u][n].z,
+                       bv[u][n].w);
+      }
+    }
+  }
+  for (; kc < c_end; ++kc) {   // remaining chunks, the last possibly partial
+    const bool in = (kc * 32 + q * 8 + 8) <= d;
+    uint4 av[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      av[h] = in ? ldg_stream(arow[h] + kc * 32) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      uint4 b = make_uint4(0, 0, 0, 0);
+      if (bval[n] && in) b = __ldg(reinterpret_cast<const uint4*>(brow[n] + kc * 32));
+      mma_bf16_16816(acc[n], av[0].x, av[1].x, av[0].y, av[1].y, b.x, b.y);
+      mma_bf16_16816(acc[n], av[0].z, av[1].z, av[0].w, av[1].w, b.z, b.w);
+    }
+  }
+
+  // partial sums -> shared memory [warp][16][EP]
+  float* part = smem + (size_t)warp * 16 * EP;
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    const int e0 = n * 8 + q * 2;
+    part[g * EP + e0] = acc[n][0];
+    part[g * EP + e0 + 1] = acc[n][1];
+    part[(g + 8) * EP + e0] = acc[n][2];
+    part[(g + 8) * EP + e0 + 1] = acc[n][3];
+  }
+  __syncthreads();
+  // logits = ((p0 + p1) + ... + p7) + bias, clamped; tile rows are LDS floats apart
+  float* tile = smem + 8 * 16 * EP;
+  const float* bias = A.bias ? A.bias + (size_t)abs_layer * E : nullptr;
+  const float big = 3.402823466e+38f;
+  for (int idx = tid; idx < 16 * EP; idx += blockDim.x) {
+    const int r = idx / EP, e = idx - r * EP;
+    float v = smem[idx];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) v = __fadd_rn(v, smem[w * 16 * EP + idx]);
+    if (bias && e < E) v = __fadd_rn(v, bias[e]);
+    tile[r * LDS + e] = fminf(fmaxf(v, -big), big);
+  }
+  __syncthreads();
+  const int rows_here = (int)min(16LL, (long long)T - tok0);
+  if (A.logits_out) {
+    float* out = A.logits_out + ((size_t)abs_layer * T + tok0) * E;
+    for (int idx = tid; idx < rows_here * E; idx += blockDim.x) {
+      const int r = idx / E, e = idx - r * E;
+      out[idx] = tile[r * LDS + e];
+    }
+  }
+  if (warp < 4) {
+    const int r = warp * 4 + (lane >> 3);
+    const long long t = tok0 + r;
+    const bool write = t < T;
+    const long long tc = write ? t : 0;
+    unsigned char* ws = A.ws + (size_t)abs_layer * A.ws_ls;
+    const int k = A.k, c = A.c;
+    const size_t lt = (size_t)abs_layer * T + tc;
+    token_epilogue_lanes8<EP>(tile + (size_t)r * LDS, lane & 7, E, k, c, A.eps_high[layer],
+                              A.t_fix[layer], A.renorm, write,
+                              reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + tc,
+                              ws + A.lay.cand_ids + (size_t)tc * c,
+                              reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)tc * c,
+                              A.expert_ids + lt * k, A.weights + lt * k);
+  }
 }
 
 }  // namespace laser

@@ -132,155 +132,6 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// Score epilogue of 4 tokens by one warp, 8 lanes per token (same arithmetic, operation by
-// operation, as token_epilogue on a shared-memory row):
-//   ranking pi by (logit desc, index asc);  e_i = exp32(x_i - x_max);
-//   Z = eight interleaved running sums a_j = sum_{i = j mod 8, ascending} e_i combined as
-//       ((a0+a1)+(a2+a3))+((a4+a5)+(a6+a7));  s = e / Z;  M_k left to right;
-//   top-k branch iff M_k >= eps_high;  otherwise c* = max(k, #{j < c : s_pi(j) >= t_fix*s_pi(0)}).
-// row: the token's logits in shared memory (nullptr-safe only through write = false with a
-// valid row).  Lane j of the group owns experts 8m + j.  All 32 lanes must call.
-template <int N>
-__device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, int E, int k, int c,
-                                                      float eps_high, float t_fix, int renorm,
-                                                      bool write, uint16_t* cstar,
-                                                      uint8_t* cand_ids, float* cand_scores,
-                                                      int32_t* expert_ids, float* weights) {
-  constexpr int EPL = N / 8;
-  const float ninf = __int_as_float(0xff800000);
-  float x[EPL];
-  float xmax = ninf;
-#pragma unroll
-  for (int m = 0; m < EPL; ++m) {
-    const int i = 8 * m + j;
-    x[m] = i < E ? row[i] : ninf;
-    xmax = fmaxf(xmax, x[m]);
-  }
-#pragma unroll
-  for (int s = 1; s < 8; s <<= 1) xmax = fmaxf(xmax, __shfl_xor_sync(0xffffffffu, xmax, s));
-  float a = 0.0f;
-#pragma unroll
-  for (int m = 0; m < EPL; ++m)
-    if (8 * m + j < E) a = __fadd_rn(a, exp32(__fsub_rn(x[m], xmax)));
-  float Z = a;
-#pragma unroll
-  for (int s = 1; s < 8; s <<= 1) Z = __fadd_rn(Z, __shfl_xor_sync(0xffffffffu, Z, s));
-
-  float prev_x = __int_as_float(0x7f800000);  // +inf
-  int prev_i = -1;
-  if (c > 32) {
-    // wide candidate lists (rare): score every rank as it is found
-    float Mk = 0.0f, thr = 0.0f;
-    int mprime = 0;
-#pragma unroll 1
-    for (int r = 0; r < c; ++r) {
-      float bx = ninf;
-      int bi = 0x7fffffff;
-#pragma unroll
-      for (int m = 0; m < EPL; ++m) {
-        const int i = 8 * m + j;
-        const float xi = x[m];
-        const bool after_prev = (xi < prev_x) || (xi == prev_x && i > prev_i);
-        if (i < E && after_prev && xi > bx) { bx = xi; bi = i; }
-      }
-#pragma unroll
-      for (int s = 1; s < 8; s <<= 1) {
-        const float ox = __shfl_xor_sync(0xffffffffu, bx, s);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
-        if (ox > bx || (ox == bx && oi < bi)) { bx = ox; bi = oi; }
-      }
-      const float sr = __fdiv_rn(exp32(__fsub_rn(bx, xmax)), Z);
-      if (r == 0) { thr = __fmul_rn(t_fix, sr); Mk = sr; }
-      else if (r < k) Mk = __fadd_rn(Mk, sr);
-      if (sr >= thr) ++mprime;
-      if (write && j == 0) {
-        cand_ids[r] = (uint8_t)bi;
-        cand_scores[r] = sr;
-        if (r < k) { expert_ids[r] = bi; weights[r] = sr; }
-      }
-      prev_x = bx;
-      prev_i = bi;
-    }
-    if (!write || j != 0) return;
-    const bool top_k_branch = (Mk >= eps_high);
-    *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
-    if (top_k_branch && renorm)
-      for (int q = 0; q < k; ++q) weights[q] = __fdiv_rn(weights[q], Mk);
-    return;
-  }
-  // ranking: c rounds of "best remaining" (local scan, then a 3-step butterfly over the group);
-  // lane j keeps the results of ranks j, j+8, j+16, j+24
-  float kx[4] = {ninf, ninf, ninf, ninf};
-  int ki[4] = {0, 0, 0, 0};
-#pragma unroll 1
-  for (int r = 0; r < c; ++r) {
-    float bx = ninf;
-    int bi = 0x7fffffff;
-#pragma unroll
-    for (int m = 0; m < EPL; ++m) {
-      const int i = 8 * m + j;
-      const float xi = x[m];
-      const bool after_prev = (xi < prev_x) || (xi == prev_x && i > prev_i);
-      if (i < E && after_prev && xi > bx) { bx = xi; bi = i; }
-    }
-#pragma unroll
-    for (int s = 1; s < 8; s <<= 1) {
-      const float ox = __shfl_xor_sync(0xffffffffu, bx, s);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
-      if (ox > bx || (ox == bx && oi < bi)) { bx = ox; bi = oi; }
-    }
-    if ((r & 7) == j) {
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if ((r >> 3) == q) { kx[q] = bx; ki[q] = bi; }
-    }
-    prev_x = bx;
-    prev_i = bi;
-  }
-  // scores of this lane's ranks
-  float sc[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    sc[q] = (8 * q + j < c) ? __fdiv_rn(exp32(__fsub_rn(kx[q], xmax)), Z) : 0.0f;
-  // M_k = s_pi(0) + ... + s_pi(k-1), left to right; rank r lives in lane r % 8, slot r / 8
-  const int gbase = (threadIdx.x & 31) & ~7;
-  float Mk = 0.0f;
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    if (8 * q < k) {   // uniform over the warp
-#pragma unroll
-      for (int l = 0; l < 8; ++l) {
-        const float v = __shfl_sync(0xffffffffu, sc[q], gbase + l);
-        const int r = 8 * q + l;
-        if (r < k) Mk = r == 0 ? v : __fadd_rn(Mk, v);
-      }
-    }
-  }
-  const float s0 = __shfl_sync(0xffffffffu, sc[0], gbase);
-  const float thr = __fmul_rn(t_fix, s0);
-  int mprime = 0;
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    if (8 * q + j < c && sc[q] >= thr) ++mprime;
-#pragma unroll
-  for (int s = 1; s < 8; s <<= 1) mprime += __shfl_xor_sync(0xffffffffu, mprime, s);
-  if (!write) return;
-  const bool top_k_branch = (Mk >= eps_high);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int r = 8 * q + j;
-    if (r < c) {
-      cand_ids[r] = (uint8_t)ki[q];
-      cand_scores[r] = sc[q];
-      if (r < k) {
-        expert_ids[r] = ki[q];
-        weights[r] = (top_k_branch && renorm) ? __fdiv_rn(sc[q], Mk) : sc[q];
-      }
-    }
-  }
-  if (j == 0) *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
-}
-
 // Router role of one block (256 threads) for tile `rt` (128 tokens) of local layer `layer`.
 // N: accumulator columns, a multiple of 16 with E <= N <= 256.
 template <int N>

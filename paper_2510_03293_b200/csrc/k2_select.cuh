@@ -69,14 +69,20 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
 __device__ __forceinline__ void st_release(int* p, int v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-// Waits until the router blocks that produce tokens [t_first, t_last] of this layer have
-// published their records.  Bounded: gives up after kK2WaitCycles and returns false.
+// Called by one full warp: waits until the router blocks that produce tokens
+// [t_first, t_last] of this layer have published their records (the lanes share the flags).
+// Bounded: gives up after kK2WaitCycles and returns false.  block = false only tests once.
 __device__ __forceinline__ bool k2_wait_ready(const int* ready, int router_rows, int t_first,
-                                              int t_last) {
+                                              int t_last, bool block = true) {
+  const int lane = threadIdx.x & 31;
+  const int rt0 = t_first / router_rows, rt1 = t_last / router_rows;
   const long long start = clock64();
-  for (int rt = t_first / router_rows; rt <= t_last / router_rows; ++rt) {
-    while (ld_acquire(ready + rt) == 0) {
-      if (clock64() - start > kK2WaitCycles) return false;
+  for (int base = rt0; base <= rt1; base += 32) {
+    const int rt = base + lane;
+    while (true) {
+      const bool set = rt > rt1 || ld_acquire(ready + rt) != 0;
+      if (__all_sync(0xffffffffu, set)) break;
+      if (!block || clock64() - start > kK2WaitCycles) return false;
       __nanosleep(100);
     }
   }
@@ -352,10 +358,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       for (int g = 0; g < n_groups && ok; ++g) {
         const int t0 = g * 32, n = min(32, T - t0);
         if (ready && (t0 % router_rows) == 0) {
-          int good = 1;
-          if (lane == 0)
-            good = k2_wait_ready(ready, router_rows, t0, min(T, t0 + router_rows) - 1) ? 1 : 0;
-          ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+          ok = k2_wait_ready(ready, router_rows, t0, min(T, t0 + router_rows) - 1);
           if (!ok) break;
         }
         for (int e = lane; e < E; e += 32) g_base[(size_t)g * E + e] = sm.L[e] - sm.Lin[e];
@@ -383,7 +386,10 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       const int t0 = b * kK2Batch, nt = min(kK2Batch, T - t0);
       if (!staged) {
         if (ready) {
-          if (tid == 0) s_flag = k2_wait_ready(ready, router_rows, t0, t0 + nt - 1) ? 1 : 0;
+          if (warp == 0) {
+            const bool good = k2_wait_ready(ready, router_rows, t0, t0 + nt - 1);
+            if (lane == 0) s_flag = good ? 1 : 0;
+          }
           __syncthreads();
           if (!s_flag) {
             if (tid == 0 && A.status) atomicOr(A.status, 2);
@@ -398,12 +404,9 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       staged = false;
       if (b + 1 < n_batches) {
         const int t1 = t0 + kK2Batch, n1 = min(kK2Batch, T - t1);
-        if (tid == 0) {
-          int okn = 1;
-          if (ready)
-            for (int rt = t1 / router_rows; rt <= (t1 + n1 - 1) / router_rows; ++rt)
-              okn &= ld_acquire(ready + rt) != 0;
-          s_flag = okn;
+        if (warp == 0) {
+          const bool okn = !ready || k2_wait_ready(ready, router_rows, t1, t1 + n1 - 1, false);
+          if (lane == 0) s_flag = okn ? 1 : 0;
         }
         __syncthreads();
         staged = s_flag != 0;

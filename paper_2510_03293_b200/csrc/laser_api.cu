@@ -127,8 +127,47 @@ bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, 
   return true;
 }
 
+// ---- split-K router for calls with few tokens ---------------------------------------------
+template <int NT, int KU, int CMAX>
+cudaError_t launch_k12_splitk(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  size_t smem = router_splitk_smem_bytes(NT);
+  const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
+  if (smem2 > smem) smem = smem2;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k12_route_select_splitk<NT, KU, CMAX>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  const unsigned tiles = (unsigned)((a.T + 15) / 16);
+  k12_route_select_splitk<NT, KU, CMAX>
+      <<<n_layers * (1 + tiles), kK2Threads, smem, s>>>(a, n_layers);
+  return cudaGetLastError();
+}
+
+template <int NT, int KU>
+cudaError_t launch_k12_splitk_for_c(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  constexpr int EP = NT * 8;
+  if (a.c <= 4) return launch_k12_splitk<NT, KU, 4>(a, n_layers, s);
+  if (a.c <= 8) return launch_k12_splitk<NT, KU, 8>(a, n_layers, s);
+  if (a.c <= 16) return launch_k12_splitk<NT, KU, (EP >= 16 ? 16 : 8)>(a, n_layers, s);
+  return launch_k12_splitk<NT, KU, (EP >= 32 ? 32 : EP)>(a, n_layers, s);
+}
+
+cudaError_t launch_k12_splitk_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  const int E = a.E;
+  if (E <= 8) return launch_k12_splitk_for_c<1, 4>(a, n_layers, s);
+  if (E <= 16) return launch_k12_splitk_for_c<2, 4>(a, n_layers, s);
+  if (E <= 32) return launch_k12_splitk_for_c<4, 4>(a, n_layers, s);
+  if (E <= 64) return launch_k12_splitk_for_c<8, 2>(a, n_layers, s);
+  if (E <= 128) return launch_k12_splitk_for_c<16, 1>(a, n_layers, s);
+  return launch_k12_splitk_for_c<32, 1>(a, n_layers, s);
+}
+
 cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
+  // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block
+  if ((long long)n_layers * ((a.T + 127) / 128) * 4 <= 148)
+    return launch_k12_splitk_for_E(a, n_layers, s);
   if (E > 32) {
     cudaError_t err = cudaSuccess;
     if (launch_k12_tensor_memory(a, n_layers, s, &err)) return err;
@@ -162,7 +201,7 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   }
   // clear the router's ready flags of these layers (one strided memset), then one launch for
   // the router and the ordered selection, one for the dispatch
-  const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 127) / 128 + 1);
+  const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 15) / 16 + 1);
   if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
                         (size_t)n, s) != cudaSuccess)
     return LASER_ERR_CUDA;

@@ -16,7 +16,7 @@ struct WorkspaceLayout {
   size_t sel_rank;     // uint8  [T, k]     rank positions chosen by the load-aware scan
   size_t grp_base;     // int32  [n_groups, E]  per-expert count of this call's assignments made
                        //                   before the group (load at group start minus L_in)
-  size_t ready;        // int32  [ceil(T/128)+1] router tiles published to the selection role
+  size_t ready;        // int32  [ceil(T/16)+1] router tiles published to the selection role
   size_t total;        // bytes per layer, multiple of 256
   int n_groups;        // ceil(T / 32): the ordered selection and the dispatch work on groups
                        // of 32 consecutive tokens
@@ -33,7 +33,7 @@ inline WorkspaceLayout make_layout(int T, int E, int k, int c) {
   w.cand_scores = off;  off = align256(off + sizeof(float) * (size_t)T * c);
   w.sel_rank = off;     off = align256(off + (size_t)T * k);
   w.grp_base = off;     off = align256(off + sizeof(int32_t) * (size_t)w.n_groups * E);
-  w.ready = off;        off = align256(off + sizeof(int32_t) * (size_t)((T + 127) / 128 + 1));
+  w.ready = off;        off = align256(off + sizeof(int32_t) * (size_t)((T + 15) / 16 + 1));
   w.total = off;
   return w;
 }

@@ -32,6 +32,14 @@ CASES = [
     (130, 512, 128, 8, 16, 0.3, 0.25, 1, 16),
     (777, 1024, 256, 8, 16, 0.30, 0.25, 1, 32),
     (100, 256, 256, 8, 40, 0.30, 0.10, 1, 32),      # candidate sets wider than a warp
+    # enough tokens for the 128-token-tile routers (fewer tokens take the split-K router)
+    (5000, 256, 8, 2, 4, 0.6, 0.5, 1, 4),
+    (5000, 256, 13, 3, 7, 0.6, 0.5, 1, 4),
+    (5000, 264, 24, 4, 9, 0.5, 0.5, 0, 3),
+    (4900, 512, 64, 6, 8, 0.40, 0.80, 0, 8),
+    (5000, 256, 100, 5, 20, 0.3, 0.3, 1, 10),
+    (5000, 256, 200, 8, 16, 0.3, 0.25, 1, 8),
+    (4800, 128, 256, 8, 40, 0.30, 0.10, 1, 32),
 ]
 
 
