@@ -22,6 +22,10 @@
  *     before returning.
  *   - Return value: LASER_OK (0) or a negative status.  On a validation error nothing is
  *     launched and no output is touched.
+ *   - The environment variable LASER_ROUTER (tile | splitk), read at every call, overrides the
+ *     choice between the 128-token-tile routers and the 16-token split-K router, which is
+ *     otherwise made from the number of tokens.  It changes speed, never results (logits may
+ *     differ in the last bits, as between any two summation orders).  Meant for tests.
  *   - Conditions only visible on the device are OR-ed into *status_word (device int32,
  *     may be NULL): LASER_DEV_LOAD_OVERFLOW, LASER_DEV_TIMEOUT.
  */

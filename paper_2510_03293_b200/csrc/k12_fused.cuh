@@ -100,7 +100,7 @@ k12_route_select_tc(const RouteArgs A, int n_layers, const __grid_constant__ CUt
   const int b = blockIdx.x - n_layers;
   const int local_layer = b % n_layers;
   const int rt = b / n_layers;
-  router_tc_block<N>(A, &map_h, &map_w, local_layer, rt, dyn_smem);
+  router_tc_block<N, (CMAX < 8 ? 8 : CMAX)>(A, &map_h, &map_w, local_layer, rt, dyn_smem);
   // router_tc_block ends with a block barrier after the last record was written
   if (threadIdx.x == 0) {
     int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +

@@ -9,10 +9,11 @@
 //   warp 1, one lane   issues four m128 x nN x k16 bf16 MMAs per stage into N fp32 columns of
 //                      tensor memory; tcgen05.commit releases the stage / publishes the tile
 //   all 8 warps        epilogue, once the accumulator is complete: the logits (+ bias) go from
-//                      tensor memory through registers into the now idle stage memory, then
-//                      groups of 8 lanes score one token each (4 tokens per warp at a time):
-//                      lane j owns the experts i = j mod 8, which makes the softmax's eight
-//                      interleaved running sums local and every reduction a 3-step butterfly.
+//                      tensor memory through registers into the now idle stage memory; then
+//                      N <= 128: warps 0..3 score one token per thread, ranking the experts
+//                      with sorting networks on 32-bit keys (token_epilogue_sorted);
+//                      N = 256: groups of 8 lanes score one token each (lane j owns the
+//                      experts i = j mod 8; every reduction is a 3-step butterfly).
 // Rows past the end of a layer and expert columns >= E hold other rows' data or zeros; they
 // are computed and ignored.  Every wait is bounded; a wait that runs out raises the timeout
 // bit, and the block still drains its copies and frees its tensor memory before it returns.
@@ -134,7 +135,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
 
 // Router role of one block (256 threads) for tile `rt` (128 tokens) of local layer `layer`.
 // N: accumulator columns, a multiple of 16 with E <= N <= 256.
-template <int N>
+template <int N, int CL>
 __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtensorMap* map_h,
                                                 const CUtensorMap* map_w, int layer, int rt,
                                                 unsigned char* dyn_smem) {
@@ -226,15 +227,62 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
     if (tid == 0 && A.status) atomicOr(A.status, 2);
   } else {
     tc_fence_after();
-    // Every stage has been read by its MMAs, so the stage memory now holds the logits tile:
-    // ROWS rows of N + 8 floats (the padding keeps the four 8-lane groups of a warp on
-    // different banks).  N = 256 does the 128 tokens in two passes of 64.
-    constexpr int LDS = N + 8;
-    constexpr int ROWS = (128 * LDS * 4 <= STAGES * STAGE_BYTES) ? 128 : 64;
-    float* tile = reinterpret_cast<float*>(stages);
+    // Every stage has been read by its MMAs, so the stage memory now holds the logits tile.
     const float big = 3.402823466e+38f;  // non-finite logits are clamped into range
     const int k = A.k, c = A.c;
     unsigned char* ws = A.ws + (size_t)abs_layer * A.ws_ls;
+    float* tile = reinterpret_cast<float*>(stages);
+    if constexpr (N <= 128) {
+      // N <= 128: all 128 rows of N + 1 floats (odd stride: a thread per row is conflict-free),
+      // then warps 0..3 score one token per thread with sorting networks
+      constexpr int LDS = N + 1;
+      static_assert(128 * LDS * 4 <= STAGES * STAGE_BYTES, "tile must fit the stage memory");
+      {
+        // tensor memory -> registers -> shared memory: warp w reads TMEM lanes 32*(w%4)..+31
+        // (its quadrant) and the column half w/4
+        const int q = warp & 3, h = warp >> 2;
+        float* dst = tile + (size_t)(q * 32 + lane) * LDS;
+        float v[32];
+#pragma unroll 1
+        for (int ch = h * (N / 64); ch < (h + 1) * (N / 64); ++ch) {
+          tc_ld32(tmem + ((uint32_t)(q * 32) << 16) + ch * 32, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int e = ch * 32 + i;
+            float xv = has_bias ? __fadd_rn(v[i], bias_s[e]) : v[i];
+            dst[e] = fminf(fmaxf(xv, -big), big);
+          }
+        }
+      }
+      __syncthreads();
+      const long long tok0 = (long long)rt * kTcTileM;
+      if (A.logits_out) {
+        const int rows_here = (int)max(0LL, min(128LL, (long long)T - tok0));
+        float* out = A.logits_out + ((size_t)abs_layer * T + tok0) * E;
+        for (int idx = tid; idx < rows_here * E; idx += blockDim.x) {
+          const int r = idx / E, e = idx - r * E;
+          out[idx] = tile[r * LDS + e];
+        }
+      }
+      const long long t = tok0 + tid;
+      if (tid < kTcTileM && t < T) {
+        const size_t lt = (size_t)abs_layer * T + t;
+        uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
+        uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
+        float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
+        if (c <= CL)
+          token_epilogue_sorted<N, CL>(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
+                                       A.t_fix[layer], A.renorm, cs_p, ids_p, sc_p,
+                                       A.expert_ids + lt * k, A.weights + lt * k);
+        else
+          token_epilogue(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer],
+                         A.renorm, cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k);
+      }
+    } else {
+    // N = 256: ROWS rows of N + 8 floats (the padding keeps the four 8-lane groups of a warp on
+    // different banks), the 128 tokens in two passes of 64; 8 lanes score one token.
+    constexpr int LDS = N + 8;
+    constexpr int ROWS = (128 * LDS * 4 <= STAGES * STAGE_BYTES) ? 128 : 64;
 #pragma unroll 1
     for (int row0 = 0; row0 < kTcTileM; row0 += ROWS) {
       // tensor memory -> registers -> shared memory: warp w reads TMEM lanes 32*(w%4)..+31
@@ -283,6 +331,7 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
       __syncthreads();   // the tile is reused by the next pass
     }
   }
+    }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

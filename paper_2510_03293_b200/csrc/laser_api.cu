@@ -3,6 +3,9 @@
 // buffer entry point), no state between calls.
 #include "../../include/laser.h"
 
+#include <cstdlib>
+#include <cstring>
+
 #include "k12_fused.cuh"
 #include "k3_dispatch.cuh"
 
@@ -165,9 +168,14 @@ cudaError_t launch_k12_splitk_for_E(const RouteArgs& a, int n_layers, cudaStream
 
 cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
-  // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block
-  if ((long long)n_layers * ((a.T + 127) / 128) * 4 <= 148)
-    return launch_k12_splitk_for_E(a, n_layers, s);
+  // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block.
+  // LASER_ROUTER=tile / splitk in the environment overrides the choice (testing aid).
+  bool few = (long long)n_layers * ((a.T + 127) / 128) * 4 <= 148;
+  if (const char* f = std::getenv("LASER_ROUTER")) {
+    if (std::strcmp(f, "tile") == 0) few = false;
+    else if (std::strcmp(f, "splitk") == 0) few = true;
+  }
+  if (few) return launch_k12_splitk_for_E(a, n_layers, s);
   if (E > 32) {
     cudaError_t err = cudaSuccess;
     if (launch_k12_tensor_memory(a, n_layers, s, &err)) return err;

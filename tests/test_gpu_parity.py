@@ -57,6 +57,13 @@ def test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B):
         assert 0.005 < frac < 0.995, f"only one branch exercised (expanded fraction {frac})"
 
 
+@pytest.mark.parametrize("T,d,E,k,c,eps,tfix,renorm,B", [c_ for c_ in CASES if c_[0] < 4000])
+def test_small_cases_through_the_tile_routers(cuda_device, monkeypatch, T, d, E, k, c, eps, tfix,
+                                              renorm, B):
+    monkeypatch.setenv("LASER_ROUTER", "tile")
+    test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B)
+
+
 def test_vanilla_and_load_only_settings(cuda_device):
     hb, wb, bias = layer(600, 512, 64, seed=5)
     z = np.zeros(64, np.int32)
@@ -218,13 +225,16 @@ def _route_layers_strided(dev, hb, wb, bias, ld_h, ld_w, k, c, eps, tfix, B):
     return r, loads, bins
 
 
+@pytest.mark.parametrize("router", ["tile", "splitk"])
 @pytest.mark.parametrize("L,T,d,E,k,c,ld_h,ld_w", [
     (3, 200, 264, 64, 6, 8, 264, 264),      # tensor-memory router: tiles straddle layers, d % 64 != 0
     (2, 333, 520, 100, 5, 12, 528, 536),    # ... with padded rows and 128 accumulator columns
     (2, 150, 256, 256, 8, 16, 320, 256),    # ... 256 accumulator columns, two-pass epilogue
     (3, 300, 264, 8, 2, 4, 272, 280),       # warp-level router with padded rows
 ])
-def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, L, T, d, E, k, c, ld_h, ld_w):
+def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, monkeypatch, router, L, T, d, E,
+                                                   k, c, ld_h, ld_w):
+    monkeypatch.setenv("LASER_ROUTER", router)   # both routers on the same small inputs
     layers = [layer(T, d, E, seed=200 + l + E, sigma=0.05) for l in range(L)]
     hb = np.stack([x[0] for x in layers]); wb = np.stack([x[1] for x in layers])
     bias = np.stack([x[2] for x in layers])
