@@ -199,12 +199,10 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
     return;   // the next batch starts with a barrier
   }
 
-  // E > 32: per (warp, expert) masks in shared memory
+  // E > 32: per (warp, expert) masks in shared memory (all zero between batches)
   uint32_t* mk = sm.mask + warp * E;
   uint8_t* ch = sm.chosen + tid * 32;
-  for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
-  __syncthreads();
-  if (valid)
+  if (valid)   // every token takes its k best to start with
     for (int j = 0; j < k; ++j) {
       ch[j] = my[j];
       atomicOr(&mk[my[j]], 1u << lane);
@@ -266,8 +264,9 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
     const int e = i % E;
     if ((i / E) * 32 < n_here) g_base[i] = sm.L[e] - sm.Lin[e] + sm.excl[i];
   }
-  __syncthreads();
+  __syncthreads();   // every thread has read the masks, excl and sm.L of this batch
   for (int e = tid; e < E; e += kK2Threads) sm.L[e] += sm.wtot[e];
+  for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
 }
 
 // Slow scan for candidate sets or k wider than a warp, or loads of 2^25 and more: one warp
@@ -313,7 +312,8 @@ __device__ __forceinline__ void k2_wide_group(int32_t* L, unsigned long long* ke
 template <int CMAX, bool SMALL>
 __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned char* k2_smem,
                                          const int* ready, int router_rows) {
-  __shared__ int s_flag;
+  __shared__ int s_flag;      // outcome of a blocking wait for the router
+  __shared__ int s_next[2];   // [b & 1]: batch b + 1 was prefetched during batch b
   const int E = A.E, k = A.k, c = A.c, T = A.T;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Ew = E > 32 ? E : 32;
@@ -341,6 +341,8 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   int32_t* g_loads = A.loads + (size_t)layer * E;
   const int n_groups = A.lay.n_groups;
 
+  if (sm.mask)
+    for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
   int too_big = 0;
   for (int e = tid; e < E; e += kK2Threads) {
     const int32_t v = g_loads[e];
@@ -381,6 +383,17 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       for (int i = tid; i < (nt * c + 15) / 16; i += kK2Threads)
         cp_async16(dst_ids + 16 * i, src_ids + 16 * i);
     };
+    // the same copy issued by the last warp alone, for the batch after the current one
+    auto stage_by_warp = [&](int b) {
+      const int t0 = b * kK2Batch, nt = min(kK2Batch, T - t0);
+      unsigned char* dst = bufs + (size_t)(b & 1) * buf_bytes;
+      const unsigned char* src_cs = reinterpret_cast<const unsigned char*>(g_cs + t0);
+      const unsigned char* src_ids = g_ids + (size_t)t0 * c;
+      unsigned char* dst_ids = dst + align256((size_t)kK2Batch * sizeof(uint16_t));
+      for (int i = lane; i < (nt * 2 + 15) / 16; i += 32) cp_async16(dst + 16 * i, src_cs + 16 * i);
+      for (int i = lane; i < (nt * c + 15) / 16; i += 32)
+        cp_async16(dst_ids + 16 * i, src_ids + 16 * i);
+    };
     bool staged = false;   // batch b is already on its way into its buffer
     for (int b = 0; b < n_batches; ++b) {
       const int t0 = b * kK2Batch, nt = min(kK2Batch, T - t0);
@@ -398,24 +411,28 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
         }
         stage(b);
       }
-      cp_async_wait_all();
-      __syncthreads();   // batch b is in shared memory; s_flag may be reused
-      // the next batch is fetched during this one if the router has already published it
-      staged = false;
-      if (b + 1 < n_batches) {
+      // The last warp looks whether the router has already published the next batch: its flag
+      // loads are issued here and first used after the barrier, so their latency is hidden.
+      const bool look = warp == kK2Warps - 1 && b + 1 < n_batches;
+      int flag_next = 1;
+      if (look && ready) {
         const int t1 = t0 + kK2Batch, n1 = min(kK2Batch, T - t1);
-        if (warp == 0) {
-          const bool okn = !ready || k2_wait_ready(ready, router_rows, t1, t1 + n1 - 1, false);
-          if (lane == 0) s_flag = okn ? 1 : 0;
-        }
-        __syncthreads();
-        staged = s_flag != 0;
-        if (staged) stage(b + 1);
+        const int rt = t1 / router_rows + lane;      // at most 16 flags per batch
+        if (rt <= (t1 + n1 - 1) / router_rows) flag_next = ld_acquire(ready + rt);
+      }
+      cp_async_wait_all();
+      __syncthreads();   // batch b is in shared memory
+      if (look) {
+        const bool okn = __all_sync(0xffffffffu, flag_next != 0);
+        if (okn) stage_by_warp(b + 1);
+        if (lane == 0) s_next[b & 1] = okn ? 1 : 0;
       }
       const unsigned char* buf = bufs + (size_t)(b & 1) * buf_bytes;
       k2_batch<CMAX, SMALL>(sm, reinterpret_cast<const uint16_t*>(buf),
                                    buf + align256((size_t)kK2Batch * sizeof(uint16_t)), nt, E, k,
                                    c, g_sel + (size_t)t0 * k, g_base + (size_t)(t0 / 32) * E);
+      // written before the barriers inside k2_batch; rewritten two batches later
+      staged = b + 1 < n_batches && s_next[b & 1] != 0;
     }
   }
   __syncthreads();
