@@ -198,6 +198,22 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- GPU arm
+def aggregate_replicas(total_ms, steps, tokens_per_rank, dist, device):
+    """Whole-job numbers of N independent replicas (the path does not shard: tokens of a layer
+    form one dependency chain).  Time is the MAX over ranks, throughput the tokens of all ranks
+    over that time.  Returns (ms_per_step, tokens_per_second)."""
+    world = 1
+    if dist is not None:
+        import torch
+
+        t = torch.tensor([float(total_ms)], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        world = dist.get_world_size()
+    ms_per_step = total_ms / steps
+    return ms_per_step, world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def run_gpu(args, w):
     import numpy as np
     import torch
@@ -263,13 +279,8 @@ def run_gpu(args, w):
     barrier()
     total_ms = t_begin.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
     tokens = L * w.T
-    value = world * tokens / (ms_per_step * 1e-3)
+    ms_per_step, value = aggregate_replicas(total_ms, args.steps, tokens, dist, dev)
 
     k1 = sum(ev[0].elapsed_time(ev[1]) for ev in stage) / args.steps
     k3 = sum(ev[2].elapsed_time(ev[3]) for ev in stage) / args.steps
