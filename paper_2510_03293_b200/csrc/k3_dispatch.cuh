@@ -1,14 +1,14 @@
 // K3: expert dispatch -- the stable grouping of pair ids t*k+j by expert -- together with the
 // final slot order, expert ids and combine weights of every token.  One warp per group of 32
-// tokens, no atomics.
+// tokens; the only atomics are warp-private shared-memory ORs.
 //
 // The ordered selection left, per group and expert, how many assignments of this call were
 // made before the group (grp_base), and the call's offsets.  A token is assigned to an expert
 // at most once, so a pair's position inside its expert's segment is
 //     grp_base[group][e] + (tokens earlier in the group that were sent to e),
-// which is also the load increment that token saw.  The warp first counts the second term for
-// all pairs of its group in pair order (match.any + warp-private running counters), then
-// every lane finishes its own token:
+// which is also the load increment that token saw.  The warp first builds, per expert, the bit
+// mask of its tokens sent there (the second term is then a population count), then every lane
+// finishes its own token:
 //   top-k branch (c* = 0): slots in score order; ids and weights were written by the router.
 //   c* > k: slots as the load-aware scan listed them (ascending load, then score rank).
 //   c* == k: the set is the k best; slots ordered by (load seen, score rank), where the load
@@ -19,9 +19,10 @@
 
 namespace laser {
 
-// Shared memory per warp: int32 base[E] | int32 pos[32*k] | uint8 pe[32*k]
+// Shared memory per warp: int32 base[E] | uint32 mask[E] | int32 pos[32*k] | uint8 pe[32*k]
 __host__ __device__ inline size_t k3_warp_smem_bytes(int E, int k) {
-  return align256(sizeof(int32_t) * (size_t)E + sizeof(int32_t) * 32 * (size_t)k + 32 * (size_t)k);
+  return align256(2 * sizeof(int32_t) * (size_t)E + sizeof(int32_t) * 32 * (size_t)k +
+                  32 * (size_t)k);
 }
 __host__ __device__ inline int k3_warps_per_block(int E, int k) {
   const size_t per = k3_warp_smem_bytes(E, k);
@@ -40,35 +41,35 @@ __global__ void k3_dispatch(const RouteArgs A) {
 
   unsigned char* mine = k3_smem + (size_t)warp * k3_warp_smem_bytes(E, k);
   int32_t* base = reinterpret_cast<int32_t*>(mine);
-  int32_t* pos = base + E;
+  uint32_t* mask = reinterpret_cast<uint32_t*>(base + E);
+  int32_t* pos = base + 2 * E;
   uint8_t* pe = reinterpret_cast<uint8_t*>(pos + 32 * k);
 
   const unsigned char* ws = A.ws + (size_t)layer * A.ws_ls;
   const long long t = (long long)g * 32 + lane;
   const bool valid = t < T;
-  const int n_here = min(32, T - g * 32);
   const int cs = valid ? reinterpret_cast<const uint16_t*>(ws + A.lay.cstar)[t] : 0;
   const uint8_t* cand = ws + A.lay.cand_ids + (size_t)t * c;
   const uint8_t* sel = ws + A.lay.sel_rank + (size_t)t * k;
   const int32_t* gb = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) + (size_t)g * E;
 
-  for (int e = lane; e < E; e += 32) base[e] = gb[e];
-  if (valid)
-    for (int j = 0; j < k; ++j) pe[lane * k + j] = cand[cs > k ? sel[j] : j];
+  for (int e = lane; e < E; e += 32) { base[e] = gb[e]; mask[e] = 0; }
   __syncwarp();
-
-  // positions inside the expert segments, in pair order
-  const int n_pairs = n_here * k;
-  for (int p0 = 0; p0 < n_pairs; p0 += 32) {
-    const int p = p0 + lane;
-    const int e = p < n_pairs ? (int)pe[p] : -1;
-    const unsigned same = __match_any_sync(0xffffffffu, e);
-    const unsigned before = same & ((1u << lane) - 1);
-    if (e >= 0) pos[p] = base[e] + __popc(before);
-    __syncwarp();
-    if (e >= 0 && before == 0) base[e] += __popc(same);
-    __syncwarp();
-  }
+  // mask[e]: which tokens of the group are sent to expert e.  A token is sent to an expert at
+  // most once, so a pair's position inside its expert's segment is the group's base count plus
+  // the number of earlier tokens of the group in that mask.
+  if (valid)
+    for (int j = 0; j < k; ++j) {
+      const uint8_t e = cand[cs > k ? sel[j] : j];
+      pe[lane * k + j] = e;
+      atomicOr(&mask[e], 1u << lane);
+    }
+  __syncwarp();
+  if (valid)
+    for (int j = 0; j < k; ++j) {
+      const int e = pe[lane * k + j];
+      pos[lane * k + j] = base[e] + __popc(mask[e] & ((1u << lane) - 1));
+    }
   if (!valid) return;
 
   const float* sc = reinterpret_cast<const float*>(ws + A.lay.cand_scores) + (size_t)t * c;
