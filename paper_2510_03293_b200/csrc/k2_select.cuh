@@ -18,6 +18,9 @@
 //             memory, and a candidate's prefix count comes back by shuffle.
 //   E  > 32   one 32-bit "who chose me" mask per (warp, expert) in shared memory, maintained
 //             with atomics by the tokens that change, and their exclusive prefix over warps.
+//             When a batch has few decision tokens, only the other tokens are counted in
+//             parallel and warp 0 takes the decision tokens one after the other
+//             (lane = candidate), which is then cheaper than block-wide sweeps.
 // The candidates' keys (load << 5 | score rank) are sorted by a compile-time bitonic network
 // over CMAX registers; the first k give the choice in the order the method lists it.
 // Per group of 32 tokens the block stores how many assignments of this call preceded the
@@ -34,6 +37,8 @@ constexpr int kK2Warps = kK2Threads / 32;
 constexpr int kK2Batch = kK2Threads;     // tokens per batch, thread = token
 constexpr int kK2FastMaxLoad = 1 << 25;  // 32-bit keys (load << 5 | rank) stay below 2^31
 constexpr int kK2MaxSweeps = kK2Batch + 2;
+constexpr int kK2ChainMax = 16;          // E > 32: batches with this many decision tokens or fewer
+                                         // take them one after the other
 constexpr long long kK2WaitCycles = 4000000000LL;  // give up a wait after ~2 s
 
 __host__ __device__ inline bool k2_fast_shape(int k, int c) { return c <= 32 && k <= 32; }
@@ -50,7 +55,9 @@ __host__ __device__ inline size_t k2_smem_bytes(int E, int c, int k) {
   size_t b = 2 * align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c) +
              align256(sizeof(int32_t) * kK2Warps * Ew);
   if (!k2_fast_shape(k, c)) return b;
-  if (E > 32) b += 2 * align256(sizeof(int32_t) * kK2Warps * E) + (size_t)kK2Batch * 32;
+  if (E > 32)
+    b += 3 * align256(sizeof(int32_t) * kK2Warps * E) + align256(sizeof(int32_t) * E) +
+         (size_t)kK2Batch * 32 + 512;
   return b + 2 * k2_batch_bytes(c);
 }
 
@@ -118,6 +125,10 @@ struct K2Smem {
   uint32_t* mask;    // [8][E]  E > 32: bit i = token i of the warp chose this expert
   int32_t* excl;     // [8][E]  E > 32: exclusive prefix of the mask popcounts over warps
   uint8_t* chosen;   // [256][32] E > 32: current choice of every token, key order
+  int32_t* dexcl;    // [8][E]  E > 32, chain mode: decisions of earlier warps per expert
+  int32_t* dcnt;     // [E]     E > 32, chain mode: decisions so far in the batch per expert
+  uint8_t* dlist;    // [256]   E > 32, chain mode: the batch's decision tokens in order
+  int32_t* dwarp;    // [8]     E > 32, chain mode: decision tokens per warp
 };
 
 // One batch of up to 256 tokens, thread = token, run by the whole block.
@@ -136,7 +147,8 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
   const bool dec = cs > k;
   const uint8_t* my = ids_s + tid * c;
   const unsigned below = (1u << lane) - 1;
-  const bool any_dec = __syncthreads_or(dec) != 0;   // also: sm.L of the previous batch is final
+  const int n_dec = __syncthreads_count(dec);   // also: sm.L of the previous batch is final
+  const bool any_dec = n_dec != 0;
   int32_t* wt = sm.wtot + warp * Ew;
 
   if (SMALL) {
@@ -202,6 +214,85 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
   // E > 32: per (warp, expert) masks in shared memory (all zero between batches)
   uint32_t* mk = sm.mask + warp * E;
   uint8_t* ch = sm.chosen + tid * 32;
+
+  // Few decision tokens: the other tokens' increments are still counted in parallel, but the
+  // decision tokens are then taken one after the other by warp 0, lane = candidate, which
+  // costs about 650 cycles each -- less than two block-wide sweeps up to kK2ChainMax tokens.
+  if (any_dec && n_dec <= kK2ChainMax) {
+    if (valid && !dec)
+      for (int j = 0; j < k; ++j) atomicOr(&mk[my[j]], 1u << lane);
+    const unsigned dmask = __ballot_sync(0xffffffffu, dec);
+    if (lane == 0) sm.dwarp[warp] = __popc(dmask);
+    for (int e = tid; e < E; e += kK2Threads) sm.dcnt[e] = 0;
+    __syncthreads();   // masks of the fixed tokens and the warps' decision counts are complete
+    if (dec) {
+      int at = __popc(dmask & below);
+      for (int w = 0; w < warp; ++w) at += sm.dwarp[w];
+      sm.dlist[at] = (uint8_t)tid;
+    }
+    for (int e = tid; e < E; e += kK2Threads) {
+      int32_t run = 0;
+#pragma unroll
+      for (int w = 0; w < kK2Warps; ++w) {
+        sm.excl[w * E + e] = run;
+        run += __popc(sm.mask[w * E + e]);
+      }
+      sm.wtot[e] = run;
+      sm.dexcl[e] = 0;   // no decision precedes warp 0
+    }
+    __syncthreads();
+    if (warp == 0) {
+      int cur_w = 0;
+      // candidate `lane` of decision token i: expert and the load it sees without the
+      // decisions of this batch; fetched one token ahead of the ranking
+      auto fetch = [&](int i, int& t, int& e, uint32_t& seen) {
+        t = sm.dlist[i];
+        const int w = t >> 5, l = t & 31;
+        const bool has = lane < (int)cs_s[t];
+        e = has ? (int)ids_s[t * c + lane] : -1;
+        seen = has ? (uint32_t)(sm.L[e] + sm.excl[w * E + e] +
+                                __popc(sm.mask[w * E + e] & ((1u << l) - 1)))
+                   : 0u;
+      };
+      int t_n, e_n;
+      uint32_t seen_n;
+      fetch(0, t_n, e_n, seen_n);
+      for (int i = 0; i < n_dec; ++i) {
+        const int t = t_n, e = e_n;
+        const uint32_t seen = seen_n;
+        if (i + 1 < n_dec) fetch(i + 1, t_n, e_n, seen_n);
+        const int w = t >> 5;
+        while (cur_w < w) {   // decisions made so far precede every token of the next warps
+          ++cur_w;
+          for (int x = lane; x < E; x += 32) sm.dexcl[cur_w * E + x] = sm.dcnt[x];
+        }
+        __syncwarp();
+        const uint32_t key = e >= 0 ? (((seen + (uint32_t)sm.dcnt[e]) << 5) | (uint32_t)lane)
+                                    : 0xffffffffu;
+        int cnt = 0;
+#pragma unroll
+        for (int j = 0; j < CMAX; ++j) cnt += __shfl_sync(0xffffffffu, key, j) < key ? 1 : 0;
+        if (e >= 0 && cnt < k) {
+          sm.dcnt[e] += 1;   // the candidates of one token are distinct experts
+          sel[t * k + cnt] = (uint8_t)lane;
+        }
+        __syncwarp();
+      }
+      while (cur_w < kK2Warps - 1) {
+        ++cur_w;
+        for (int x = lane; x < E; x += 32) sm.dexcl[cur_w * E + x] = sm.dcnt[x];
+      }
+    }
+    __syncthreads();
+    for (int i = tid; i < kK2Warps * E; i += kK2Threads) {
+      const int e = i % E;
+      if ((i / E) * 32 < n_here) g_base[i] = sm.L[e] - sm.Lin[e] + sm.excl[i] + sm.dexcl[i];
+    }
+    __syncthreads();   // every thread has read the masks, excl, dexcl and sm.L of this batch
+    for (int e = tid; e < E; e += kK2Threads) sm.L[e] += sm.wtot[e] + sm.dcnt[e];
+    for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
+    return;
+  }
   if (valid)   // every token takes its k best to start with
     for (int j = 0; j < k; ++j) {
       ch[j] = my[j];
@@ -325,10 +416,15 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   sm.keys = reinterpret_cast<unsigned long long*>(p);  p += align256(sizeof(unsigned long long) * c);
   sm.wtot = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * kK2Warps * Ew);
   sm.mask = nullptr; sm.excl = nullptr; sm.chosen = nullptr;
+  sm.dexcl = nullptr; sm.dcnt = nullptr; sm.dlist = nullptr; sm.dwarp = nullptr;
   if (E > 32 && k2_fast_shape(k, c)) {
     sm.mask = reinterpret_cast<uint32_t*>(p);  p += align256(sizeof(int32_t) * kK2Warps * E);
     sm.excl = reinterpret_cast<int32_t*>(p);   p += align256(sizeof(int32_t) * kK2Warps * E);
     sm.chosen = p;                              p += (size_t)kK2Batch * 32;
+    sm.dexcl = reinterpret_cast<int32_t*>(p);  p += align256(sizeof(int32_t) * kK2Warps * E);
+    sm.dcnt = reinterpret_cast<int32_t*>(p);   p += align256(sizeof(int32_t) * E);
+    sm.dlist = p;                               p += 256;
+    sm.dwarp = reinterpret_cast<int32_t*>(p);  p += 256;
   }
   unsigned char* bufs = p;
   const size_t buf_bytes = k2_batch_bytes(c);
