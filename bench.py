@@ -296,7 +296,7 @@ def run_gpu(args, w):
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate and scores",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "accumulate": "f32 (logits, scores and weights in f32; ids, loads, dispatch in int32)",
         "data": "synthetic", "config": workload_config(w, L, n_copies),
         "roofline": {"bound": "hbm", "kernel": router_kernel_name(w, L),
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
@@ -411,7 +411,7 @@ def run_decode(args, w):
         "metric": METRIC, "value": tokens / (ms_graph * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_graph,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 inputs, f32 accumulate and scores", "data": "synthetic",
+        "dtype": "bf16", "accumulate": "f32 (logits, scores and weights in f32; ids, loads, dispatch in int32)", "data": "synthetic",
         "config": {"workload": "decode: %d successive calls x T=%d, d=%d bf16, E=%d, k=%d, c=%d, "
                                "loads carried across calls" % (S, w.T, w.d, w.E, w.k, w.c),
                    "tokens_per_step": tokens,
