@@ -249,3 +249,32 @@ def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, monkeypatch, rou
         assert np.isfinite(g["logits"]).all()
         check_against_oracle(g, hb[l], wb[l], bias[l], np.zeros(E, np.int32), k, c, 0.5, 0.5, 1, B,
                              bins0=np.zeros(B, np.int32))
+
+
+def test_more_layers_than_one_launch_holds(cuda_device):
+    """70 layers: the library routes them in groups of 64 layers per launch."""
+    import torch
+
+    from paper_2510_03293_b200 import laser
+
+    dev = cuda_device
+    Lr, T, d, E, k, c, B = 70, 40, 64, 8, 2, 4, 2
+    layers = [layer(T, d, E, seed=300 + l, sigma=0.2) for l in range(Lr)]
+    hb = np.stack([x[0] for x in layers]); wb = np.stack([x[1] for x in layers])
+    bias = np.stack([x[2] for x in layers])
+    eps = [0.55 + 0.002 * l for l in range(Lr)]
+    p = laser.make_params(T, d, E, k, c, 0.0, 0.5, 1, B)
+    loads = torch.zeros((Lr, E), dtype=torch.int32, device=dev)
+    bins = torch.zeros((Lr, B), dtype=torch.int32, device=dev)
+    r = laser.route_layers(to_dev_bf16(hb, dev), to_dev_bf16(wb, dev),
+                           torch.from_numpy(bias).to(dev), loads, p, bin_loads=bins, eps_high=eps,
+                           want_logits=True)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    for l in (0, 1, 63, 64, 69):
+        g = dict(expert_ids=r.expert_ids[l].cpu().numpy(), weights=r.weights[l].cpu().numpy(),
+                 offsets=r.offsets[l].cpu().numpy(), perm=r.perm[l].cpu().numpy(),
+                 loads=loads[l].cpu().numpy(), bin_loads=bins[l].cpu().numpy(),
+                 logits=r.logits[l].cpu().numpy(), status=0)
+        check_against_oracle(g, hb[l], wb[l], bias[l], np.zeros(E, np.int32), k, c, eps[l], 0.5, 1,
+                             B, bins0=np.zeros(B, np.int32))
