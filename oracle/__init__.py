@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.lo_softmax.restype = None
         L.lo_route.argtypes = [vp, i32, i32, i32, i32, f32, f32, i32, vp, vp, vp, vp]
         L.lo_route.restype = i32
+        L.lo_route_relaxed.argtypes = [vp, i32, i32, i32, i32, f32, f32, i32, i32, vp, vp, vp, vp]
+        L.lo_route_relaxed.restype = i32
         L.lo_topk.argtypes = [vp, i32, i32, i32, vp]
         L.lo_topk.restype = None
         L.lo_dispatch.argtypes = [vp, i32, i32, i32, vp, vp]
@@ -113,6 +115,24 @@ def route(x: np.ndarray, loads: np.ndarray, k: int, c: int, eps_high: float, t_f
     return ids, w, L, cs
 
 
+def route_relaxed(x: np.ndarray, loads: np.ndarray, k: int, c: int, eps_high: float,
+                  t_fix: float, granularity: int, renormalize: bool = True):
+    """The RELAXED load update (not the method's rule): a token sees the loads as they stood
+    at the start of its chunk of ``granularity`` tokens (0 = one snapshot per call).  Same
+    return values as ``route``; ``granularity = 1`` is ``route``."""
+    x = _c(x, np.float32)
+    T, E = x.shape
+    L = _c(loads, np.int32).copy()
+    ids = np.empty((T, k), np.int32)
+    w = np.empty((T, k), np.float32)
+    cs = np.empty((T,), np.int32)
+    rc = lib().lo_route_relaxed(_p(x), T, E, k, c, eps_high, t_fix, int(bool(renormalize)),
+                                int(granularity), _p(L), _p(ids), _p(w), _p(cs))
+    if rc != 0:
+        raise ValueError("lo_route_relaxed rejected its arguments")
+    return ids, w, L, cs
+
+
 def topk(x: np.ndarray, k: int) -> np.ndarray:
     x = _c(x, np.float32)
     T, E = x.shape
@@ -140,12 +160,16 @@ def bins(counts: np.ndarray, expert_to_bin: np.ndarray, bin_loads: np.ndarray) -
 
 
 def route_full(hidden_bits, wg_bits, bias, loads, expert_to_bin, bin_loads,
-               k, c, eps_high, t_fix, renormalize=True, x=None):
-    """Whole path: logits (unless given) -> routing -> dispatch -> bins.  Dict of arrays."""
+               k, c, eps_high, t_fix, renormalize=True, x=None, granularity=1):
+    """Whole path: logits (unless given) -> routing -> dispatch -> bins.  Dict of arrays.
+    ``granularity != 1`` selects the relaxed load update of ``route_relaxed``."""
     if x is None:
         x = logits(hidden_bits, wg_bits, bias)
     E = x.shape[1]
-    ids, w, L, cs = route(x, loads, k, c, eps_high, t_fix, renormalize)
+    if granularity == 1:
+        ids, w, L, cs = route(x, loads, k, c, eps_high, t_fix, renormalize)
+    else:
+        ids, w, L, cs = route_relaxed(x, loads, k, c, eps_high, t_fix, granularity, renormalize)
     offsets, perm = dispatch(ids, E)
     counts = (L - np.asarray(loads, np.int32)).astype(np.int32)
     out = dict(logits=x, expert_ids=ids, weights=w, loads=L, cstar=cs,

@@ -187,6 +187,70 @@ int32_t lo_route(const float* x, int32_t T, int32_t E, int32_t k, int32_t c,
 }
 
 /*
+ * RELAXED variant of the load update -- not the method's rule, kept apart from lo_route and
+ * only ever reported beside it.  The text says loads are tracked "per token and per batch";
+ * the reading taken for the method is "after every token" (lo_route).  Here the loads that a
+ * token SEES are refreshed only every G tokens: tokens are cut into chunks of G consecutive
+ * rows, and every token of a chunk ranks its candidates by the loads as they stood when the
+ * chunk began (G = 0: one chunk per call, i.e. a per-call snapshot).  The counters themselves
+ * still grow by one per assignment.  G = 1 is lo_route.  Everything else (softmax, top-k
+ * mass test, pool, trimming, tie-breaks, weights) is as in lo_route.
+ */
+int32_t lo_route_relaxed(const float* x, int32_t T, int32_t E, int32_t k, int32_t c,
+                         float eps_high, float t_fix, int32_t renormalize, int32_t G,
+                         int32_t* loads, int32_t* ids, float* weights, int32_t* cstar) {
+    if (T < 0 || E < 1 || k < 1 || k > c || c > E || G < 0) return -1;
+    float* s = (float*)malloc(sizeof(float) * (size_t)E);
+    ranked_t* pi = (ranked_t*)malloc(sizeof(ranked_t) * (size_t)E);
+    int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)E);
+    int32_t* seen = (int32_t*)malloc(sizeof(int32_t) * (size_t)E);   /* loads at chunk start */
+    if (!s || !pi || !cand || !seen) { free(s); free(pi); free(cand); free(seen); return -1; }
+
+    for (int32_t t = 0; t < T; ++t) {
+        if (G == 0 ? t == 0 : t % G == 0) memcpy(seen, loads, sizeof(int32_t) * (size_t)E);
+        const float* xt = x + (int64_t)t * E;
+        lo_softmax(xt, E, s);
+        for (int32_t e = 0; e < E; ++e) { pi[e].x = xt[e]; pi[e].e = e; }
+        qsort(pi, (size_t)E, sizeof(ranked_t), rank_cmp);
+
+        float Mk = s[pi[0].e];
+        for (int32_t j = 1; j < k; ++j) Mk = Mk + s[pi[j].e];
+
+        int32_t* A = ids + (int64_t)t * k;
+        if (Mk >= eps_high) {
+            for (int32_t j = 0; j < k; ++j) A[j] = pi[j].e;
+            if (cstar) cstar[t] = 0;
+        } else {
+            float thr = t_fix * s[pi[0].e];
+            int32_t mprime = 0;
+            for (int32_t j = 0; j < c; ++j) if (s[pi[j].e] >= thr) ++mprime;
+            int32_t cs = mprime > k ? mprime : k;
+            for (int32_t j = 0; j < cs; ++j) {   /* insertion sort by (load seen, rank) */
+                int32_t pos = j;
+                while (pos > 0 && seen[pi[cand[pos - 1]].e] > seen[pi[j].e]) {
+                    cand[pos] = cand[pos - 1];
+                    --pos;
+                }
+                cand[pos] = j;
+            }
+            for (int32_t j = 0; j < k; ++j) A[j] = pi[cand[j]].e;
+            if (cstar) cstar[t] = cs;
+        }
+
+        float* w = weights + (int64_t)t * k;
+        for (int32_t j = 0; j < k; ++j) w[j] = s[A[j]];
+        if (renormalize) {
+            float sum = w[0];
+            for (int32_t j = 1; j < k; ++j) sum = sum + w[j];
+            for (int32_t j = 0; j < k; ++j) w[j] = w[j] / sum;
+        }
+        for (int32_t j = 0; j < k; ++j) loads[A[j]] += 1;
+    }
+    free(s); free(pi); free(cand); free(seen);
+    return 0;
+}
+
+/*
  * Vanilla top-k routing (Introduction: "selects the k experts with the highest scores";
  * the Baselines paragraph).  Written independently of lo_route: k rounds of argmax over
  * the logits with already-taken experts masked out; ties go to the lower index.

@@ -268,3 +268,67 @@ def test_workload_parameters_come_from_the_papers_table():
     assert w["stress"].t_fix == min(min(v[0]) for v in table.values())
     assert [w["mixtral"].eps_for_layer(l) for l in (0, 10, 11, 21, 22, 31)] == \
         [mix[1][0], mix[1][0], mix[1][1], mix[1][1], mix[1][2], mix[1][2]]
+
+
+# ---- relaxed load update (reported beside the method's rule, never instead of it) -----------
+def _rand_logits(T, E, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    return (rng.standard_normal((T, E)) * scale).astype(np.float32)
+
+
+def test_relaxed_with_granularity_one_is_the_rule():
+    x = _rand_logits(700, 8, 1)
+    L0 = np.array([3, 0, 2, 5, 1, 1, 0, 4], np.int32)
+    a = oracle.route(x, L0, 2, 4, 0.64, 0.6)
+    b = oracle.route_relaxed(x, L0, 2, 4, 0.64, 0.6, 1)
+    for u, v in zip(a, b):
+        assert np.array_equal(u, v)
+
+
+def test_relaxed_snapshot_equals_any_chunk_longer_than_the_call():
+    x = _rand_logits(300, 16, 2, 0.3)
+    L0 = np.arange(16, dtype=np.int32) % 5
+    a = oracle.route_relaxed(x, L0, 3, 8, 0.9, 0.2, 0)
+    for G in (300, 301, 4096):
+        b = oracle.route_relaxed(x, L0, 3, 8, 0.9, 0.2, G)
+        for u, v in zip(a, b):
+            assert np.array_equal(u, v)
+    assert int((a[2] - L0).sum()) == 300 * 3
+
+
+def test_relaxed_snapshot_from_equal_loads_sends_every_token_to_its_top_k():
+    # all loads equal on entry and never refreshed: ties go by score, so every token takes its
+    # k best -- the reason a per-call snapshot cannot be what the paper means by load-aware
+    x = _rand_logits(200, 8, 3, 0.2)
+    ids, _, L, cs = oracle.route_relaxed(x, np.full(8, 7, np.int32), 2, 6, 2.0, 0.0, 0)
+    assert np.all(cs == 6)
+    assert np.array_equal(np.sort(ids, 1), np.sort(oracle.topk(x, 2), 1))
+
+
+def test_relaxed_chunks_by_hand():
+    # E = 3, k = 1, every token expands over all 3 experts with equal scores; G = 2:
+    # chunk 0 (loads 0,0,0): both tokens pick expert 0; chunk 1 (2,0,0): both pick expert 1;
+    # chunk 2 (2,2,0): both pick expert 2.  The rule itself would cycle 0,1,2,0,1,2.
+    x = np.zeros((6, 3), np.float32)
+    ids, _, L, _ = oracle.route_relaxed(x, np.zeros(3, np.int32), 1, 3, 2.0, 0.0, 2)
+    assert ids[:, 0].tolist() == [0, 0, 1, 1, 2, 2] and L.tolist() == [2, 2, 2]
+    ids1, _, _, _ = oracle.route(x, np.zeros(3, np.int32), 1, 3, 2.0, 0.0)
+    assert ids1[:, 0].tolist() == [0, 1, 2, 0, 1, 2]
+
+
+def test_relaxed_matches_a_python_restatement():
+    x = _rand_logits(150, 8, 4, 0.4)
+    L0 = np.array([0, 2, 0, 1, 0, 0, 3, 0], np.int32)
+    k, c, eps, tf, G = 2, 5, 0.7, 0.4, 32
+    ids, _, L, _ = oracle.route_relaxed(x, L0, k, c, eps, tf, G)
+    S = oracle.softmax(x)
+    loads = [int(v) for v in L0]
+    seen = list(loads)
+    for t in range(150):
+        if t % G == 0:
+            seen = list(loads)
+        A, _, _ = lit.alg1_token(S[t], seen, k, c, eps, tf, x[t])
+        assert list(ids[t]) == list(A), t
+        for e in A:
+            loads[e] += 1
+    assert loads == L.tolist()
