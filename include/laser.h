@@ -74,7 +74,13 @@ enum { LASER_MAX_EXPERTS = 256 };
  *                (pool = the c best).  eps_high > 1, t_fix = 0, c = E is load-only routing.
  *   trim_mode    0 = TOP (keep the c best).  1 = RANDOM is not implemented
  *                (LASER_ERR_UNSUPPORTED).
- *   update_granularity  1 = loads are updated after every token (the only mode).
+ *   update_granularity  1 = the loads a token sees include every earlier token (the method's
+ *                rule as this library reads it, and the default of every helper).
+ *                0 or a multiple of 32 = RELAXED variant, not the rule and never chosen for
+ *                the caller: the loads seen are refreshed only every G tokens (0: once per
+ *                call).  It needs no iteration to stay exact to its own definition and is
+ *                there to study how far coarser updates drift.  Other values:
+ *                LASER_ERR_UNSUPPORTED.
  *   renormalize  1: combine weights are divided by their sum over the k chosen experts;
  *                0: raw softmax scores.
  *   n_bins       number of device bins B >= 1 (only used when bin_loads != NULL)

@@ -52,7 +52,7 @@ __host__ __device__ inline size_t k2_batch_bytes(int c) {
 //   2 batch buffers (c*, candidate ids)
 __host__ __device__ inline size_t k2_smem_bytes(int E, int c, int k) {
   const size_t Ew = E > 32 ? E : 32;
-  size_t b = 2 * align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c) +
+  size_t b = 3 * align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c) +
              align256(sizeof(int32_t) * kK2Warps * Ew);
   if (!k2_fast_shape(k, c)) return b;
   if (E > 32)
@@ -120,6 +120,8 @@ __device__ __forceinline__ void sort_keys(uint32_t (&a)[N]) {
 struct K2Smem {
   int32_t* L;        // [E] loads at the start of the current batch
   int32_t* Lin;      // [E] loads on entry
+  int32_t* Lvis;     // [E] relaxed variant: loads at the start of the chunk that reaches
+                     //     into the current batch from an earlier one
   unsigned long long* keys;  // [c] slow scan only
   int32_t* wtot;     // [8][max(E,32)] per warp and expert: tokens of the warp that chose it
   uint32_t* mask;    // [8][E]  E > 32: bit i = token i of the warp chose this expert
@@ -139,9 +141,17 @@ struct K2Smem {
 template <int CMAX, bool SMALL>
 __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
                                          const uint8_t* ids_s, int n_here, int E, int k, int c,
-                                         uint8_t* sel, int32_t* g_base) {
+                                         uint8_t* sel, int32_t* g_base, int G, int t0) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Ew = E > 32 ? E : 32;
+  // Relaxed variant (G != 1; G is 0 or a multiple of 32, so a warp's 32 tokens share a chunk):
+  // a token sees the loads at the start of its chunk.  If the chunk began in an earlier batch
+  // those are sm.Lvis and nothing of this batch; otherwise sm.L plus the choices of the warps
+  // before the chunk's first warp wc.
+  const bool strict = G == 1;
+  const int c0 = G == 0 ? 0 : ((t0 + warp * 32) / (G > 0 ? G : 1)) * G;   // chunk start (token)
+  const bool outside = !strict && c0 < t0;
+  const int wc = (strict || outside) ? 0 : (c0 - t0) / 32;
   const bool valid = tid < n_here;
   const int cs = valid ? cs_s[tid] : 0;
   const bool dec = cs > k;
@@ -163,7 +173,7 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
 #pragma unroll
       for (int r = 0; r < CMAX; ++r) {
         cid[r] = (dec && r < cs) ? my[r] : 0;
-        Lc[r] = (uint32_t)sm.L[cid[r]];
+        Lc[r] = (uint32_t)(outside ? sm.Lvis[cid[r]] : sm.L[cid[r]]);
       }
     }
     for (int sweep = 0; sweep < kK2MaxSweeps; ++sweep) {
@@ -174,15 +184,20 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
       wt[lane] = __popc(Bm);
       __syncthreads();
       excl = 0;
-      for (int w = 0; w < warp; ++w) excl += sm.wtot[w * Ew + lane];
+      int32_t exv = 0;   // relaxed: choices of the warps before the chunk's first warp
+      for (int w = 0; w < warp; ++w) {
+        const int32_t v = sm.wtot[w * Ew + lane];
+        excl += v;
+        if (w < wc) exv += v;
+      }
       if (!any_dec) break;
       uint32_t m_new = m;
 #pragma unroll
       for (int r = 0; r < CMAX; ++r) {
         const uint32_t Br = __shfl_sync(0xffffffffu, Bm, cid[r]);
-        const uint32_t ex = (uint32_t)__shfl_sync(0xffffffffu, excl, cid[r]);
-        key[r] = (dec && r < cs) ? (((Lc[r] + ex + __popc(Br & below)) << 5) | (uint32_t)r)
-                                 : 0xffffffffu;
+        const uint32_t ex = (uint32_t)__shfl_sync(0xffffffffu, strict ? excl : exv, cid[r]);
+        const uint32_t seen = Lc[r] + ex + (strict ? (uint32_t)__popc(Br & below) : 0u);
+        key[r] = (dec && r < cs) ? ((seen << 5) | (uint32_t)r) : 0xffffffffu;
       }
       if (dec) {
         sort_keys<CMAX>(key);
@@ -202,10 +217,19 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
     }
     if (lane < E && warp * 32 < n_here)
       g_base[warp * E + lane] = sm.L[lane] - sm.Lin[lane] + excl;
-    __syncthreads();   // every thread has read sm.L and wtot
+    __syncthreads();   // every thread has read sm.L, sm.Lvis and wtot
     if (warp == 0 && lane < E) {
-      int32_t tot = 0;
-      for (int w = 0; w < kK2Warps; ++w) tot += sm.wtot[w * Ew + lane];
+      // relaxed: the chunk that holds the next batch's first token, if it began in this batch
+      const int t_next = t0 + kK2Batch;
+      const int c_next = G == 0 ? 0 : (t_next / (G > 0 ? G : 1)) * G;
+      const int wl = (c_next - t0) / 32;
+      int32_t tot = 0, upto = 0;
+      for (int w = 0; w < kK2Warps; ++w) {
+        const int32_t v = sm.wtot[w * Ew + lane];
+        tot += v;
+        if (w < wl) upto += v;
+      }
+      if (!strict && c_next >= t0) sm.Lvis[lane] = sm.L[lane] + (c_next < t_next ? upto : tot);
       sm.L[lane] += tot;
     }
     return;   // the next batch starts with a barrier
@@ -218,7 +242,7 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
   // Few decision tokens: the other tokens' increments are still counted in parallel, but the
   // decision tokens are then taken one after the other by warp 0, lane = candidate, which
   // costs about 650 cycles each -- less than two block-wide sweeps up to kK2ChainMax tokens.
-  if (any_dec && n_dec <= kK2ChainMax) {
+  if (strict && any_dec && n_dec <= kK2ChainMax) {
     if (valid && !dec)
       for (int j = 0; j < k; ++j) atomicOr(&mk[my[j]], 1u << lane);
     const unsigned dmask = __ballot_sync(0xffffffffu, dec);
@@ -304,7 +328,7 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
 #pragma unroll
     for (int r = 0; r < CMAX; ++r) {
       cid[r] = (dec && r < cs) ? my[r] : 0;
-      Lc[r] = (uint32_t)sm.L[cid[r]];
+      Lc[r] = (uint32_t)(outside ? sm.Lvis[cid[r]] : sm.L[cid[r]]);
     }
   }
   for (int sweep = 0; sweep < kK2MaxSweeps; ++sweep) {
@@ -324,8 +348,11 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
     if (dec) {
 #pragma unroll
       for (int r = 0; r < CMAX; ++r)
-        key[r] = r < cs ? (((Lc[r] + (uint32_t)sm.excl[warp * E + cid[r]] +
-                             __popc(mk[cid[r]] & below)) << 5) | (uint32_t)r)
+        key[r] = r < cs ? (((Lc[r] +
+                             (strict ? (uint32_t)sm.excl[warp * E + cid[r]] +
+                                           (uint32_t)__popc(mk[cid[r]] & below)
+                                     : (outside ? 0u : (uint32_t)sm.excl[wc * E + cid[r]])))
+                            << 5) | (uint32_t)r)
                         : 0xffffffffu;
       sort_keys<CMAX>(key);
 #pragma unroll
@@ -355,14 +382,24 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
     const int e = i % E;
     if ((i / E) * 32 < n_here) g_base[i] = sm.L[e] - sm.Lin[e] + sm.excl[i];
   }
-  __syncthreads();   // every thread has read the masks, excl and sm.L of this batch
-  for (int e = tid; e < E; e += kK2Threads) sm.L[e] += sm.wtot[e];
+  __syncthreads();   // every thread has read the masks, excl, sm.L and sm.Lvis of this batch
+  {
+    const int t_next = t0 + kK2Batch;
+    const int c_next = G == 0 ? 0 : (t_next / (G > 0 ? G : 1)) * G;
+    const int wl = (c_next - t0) / 32;
+    for (int e = tid; e < E; e += kK2Threads) {
+      if (!strict && c_next >= t0)
+        sm.Lvis[e] = sm.L[e] + (c_next < t_next ? sm.excl[wl * E + e] : sm.wtot[e]);
+      sm.L[e] += sm.wtot[e];
+    }
+  }
   for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
 }
 
 // Slow scan for candidate sets or k wider than a warp, or loads of 2^25 and more: one warp
 // walks every token of one group; 64-bit keys (load, score rank) go through shared memory.
-__device__ __forceinline__ void k2_wide_group(int32_t* L, unsigned long long* keys,
+__device__ __forceinline__ void k2_wide_group(int32_t* L, const int32_t* Lsee,
+                                              unsigned long long* keys,
                                               const uint16_t* g_cs, const uint8_t* g_ids,
                                               uint8_t* g_sel, int ntok, int k, int c, int lane) {
   for (long long t = 0; t < ntok; ++t) {
@@ -372,7 +409,7 @@ __device__ __forceinline__ void k2_wide_group(int32_t* L, unsigned long long* ke
       for (int j = lane; j < k; j += 32) L[ids[j]] += 1;
     } else {
       for (int j = lane; j < cs; j += 32)
-        keys[j] = (((unsigned long long)(uint32_t)L[ids[j]]) << 8) | (unsigned)j;
+        keys[j] = (((unsigned long long)(uint32_t)Lsee[ids[j]]) << 8) | (unsigned)j;
       __syncwarp();
       unsigned chosen = 0;
       int it = 0;
@@ -413,6 +450,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   unsigned char* p = k2_smem;
   sm.L = reinterpret_cast<int32_t*>(p);       p += align256(sizeof(int32_t) * E);
   sm.Lin = reinterpret_cast<int32_t*>(p);     p += align256(sizeof(int32_t) * E);
+  sm.Lvis = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * E);
   sm.keys = reinterpret_cast<unsigned long long*>(p);  p += align256(sizeof(unsigned long long) * c);
   sm.wtot = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * kK2Warps * Ew);
   sm.mask = nullptr; sm.excl = nullptr; sm.chosen = nullptr;
@@ -444,6 +482,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
     const int32_t v = g_loads[e];
     sm.L[e] = v;
     sm.Lin[e] = v;
+    sm.Lvis[e] = v;
     // a counter within T of 2^31-1 could wrap during the call: raise the status bit
     if (v < 0 || v > 0x7fffffff - T) { if (A.status) atomicOr(A.status, 1); }
     if (v < 0 || v > kK2FastMaxLoad - T) too_big = 1;
@@ -460,8 +499,12 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
           if (!ok) break;
         }
         for (int e = lane; e < E; e += 32) g_base[(size_t)g * E + e] = sm.L[e] - sm.Lin[e];
-        k2_wide_group(sm.L, sm.keys, g_cs + t0, g_ids + (size_t)t0 * c, g_sel + (size_t)t0 * k, n,
-                      k, c, lane);
+        if (A.G != 1 && (A.G == 0 ? t0 == 0 : t0 % A.G == 0)) {   // relaxed: a chunk begins
+          for (int e = lane; e < E; e += 32) sm.Lvis[e] = sm.L[e];
+          __syncwarp();
+        }
+        k2_wide_group(sm.L, A.G == 1 ? sm.L : sm.Lvis, sm.keys, g_cs + t0, g_ids + (size_t)t0 * c,
+                      g_sel + (size_t)t0 * k, n, k, c, lane);
       }
       if (!ok && lane == 0 && A.status) atomicOr(A.status, 2);
     }
@@ -526,7 +569,8 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       const unsigned char* buf = bufs + (size_t)(b & 1) * buf_bytes;
       k2_batch<CMAX, SMALL>(sm, reinterpret_cast<const uint16_t*>(buf),
                                    buf + align256((size_t)kK2Batch * sizeof(uint16_t)), nt, E, k,
-                                   c, g_sel + (size_t)t0 * k, g_base + (size_t)(t0 / 32) * E);
+                                   c, g_sel + (size_t)t0 * k, g_base + (size_t)(t0 / 32) * E, A.G,
+                                   t0);
       // written before the barriers inside k2_batch; rewritten two batches later
       staged = b + 1 < n_batches && s_next[b & 1] != 0;
     }

@@ -97,14 +97,21 @@ __global__ void k3_dispatch(const RouteArgs A) {
     }
   } else {
     // load seen by rank j: L_in[e] + position; L_in = L_out - count.  Smaller (load, j) first.
+    // (Relaxed variant: the assignments made before the token's chunk take the position's place.)
     const int32_t* Lout = A.loads + (size_t)layer * E;
+    const int32_t* gb0 = nullptr;
+    if (A.G != 1)
+      gb0 = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) +
+            (size_t)(A.G == 0 ? 0 : ((t / A.G) * A.G) / 32) * E;
     for (int j = 0; j < k; ++j) {
       const int ej = mype[j];
-      const long long Lj = (long long)Lout[ej] - (off[ej + 1] - off[ej]) + mypos[j];
+      const long long Lj = (long long)Lout[ej] - (off[ej + 1] - off[ej]) +
+                           (gb0 ? gb0[ej] : mypos[j]);
       int slot = 0;
       for (int i = 0; i < k; ++i) {
         const int ei = mype[i];
-        const long long Li = (long long)Lout[ei] - (off[ei + 1] - off[ei]) + mypos[i];
+        const long long Li = (long long)Lout[ei] - (off[ei + 1] - off[ei]) +
+                             (gb0 ? gb0[ei] : mypos[i]);
         slot += (Li < Lj || (Li == Lj && i < j)) ? 1 : 0;
       }
       ids[slot] = ej;

@@ -24,7 +24,8 @@ int validate_params(const laser_params* p) {
     return LASER_ERR_INVALID_ARG;
   if (p->trim_mode == 1) return LASER_ERR_UNSUPPORTED;
   if (p->trim_mode != 0) return LASER_ERR_INVALID_ARG;
-  if (p->update_granularity != 1) return LASER_ERR_UNSUPPORTED;
+  if (p->update_granularity < 0) return LASER_ERR_INVALID_ARG;
+  if (p->update_granularity != 1 && p->update_granularity % 32 != 0) return LASER_ERR_UNSUPPORTED;
   if (p->n_bins < 1) return LASER_ERR_INVALID_ARG;
   if (p->ld_hidden < p->d || p->ld_w < p->d) return LASER_ERR_INVALID_ARG;
   if (p->ld_hidden % 8 != 0 || p->ld_w % 8 != 0) return LASER_ERR_MISALIGNED;
@@ -296,6 +297,7 @@ extern "C" int laser_route_layers_profiled(
   a.lay = lay;
   a.T = p->T; a.d = p->d; a.E = p->E; a.k = p->k; a.c = p->c;
   a.n_bins = p->n_bins; a.renorm = p->renormalize ? 1 : 0;
+  a.G = p->update_granularity;
   a.ld_h = p->ld_hidden; a.ld_w = p->ld_w;
 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

@@ -55,6 +55,9 @@ struct RouteArgs {
   unsigned char* ws;       size_t ws_ls;          // bytes
   WorkspaceLayout lay;
   int T, d, E, k, c, n_bins, renorm;
+  int G;                   // load-update granularity: 1 = after every token (the rule);
+                           // 0 or a multiple of 32 = relaxed variant (loads seen refreshed
+                           // every G tokens, 0 = once per call)
   long long ld_h, ld_w;
   int layer0;              // first layer of this launch
   float eps_high[kMaxLayersPerLaunch];

@@ -50,7 +50,8 @@ def good(**over):
     (dict(ld_hidden=260), laser.ERR_MISALIGNED),
     (dict(trim_mode=1), laser.ERR_UNSUPPORTED),
     (dict(trim_mode=7), laser.ERR_INVALID_ARG),
-    (dict(update_granularity=0), laser.ERR_UNSUPPORTED),
+    (dict(update_granularity=7), laser.ERR_UNSUPPORTED),
+    (dict(update_granularity=-32), laser.ERR_INVALID_ARG),
     (dict(T=2**30, k=4, c=4), laser.ERR_INVALID_ARG),
 ])
 def test_bad_parameters_are_rejected(over, status):

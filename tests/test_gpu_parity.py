@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 
 from paper_2510_03293_b200 import synth
+import oracle
 from gpu_util import check_against_oracle, run_gpu, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
@@ -278,3 +279,49 @@ def test_more_layers_than_one_launch_holds(cuda_device):
                  logits=r.logits[l].cpu().numpy(), status=0)
         check_against_oracle(g, hb[l], wb[l], bias[l], np.zeros(E, np.int32), k, c, eps[l], 0.5, 1,
                              B, bins0=np.zeros(B, np.int32))
+
+
+# ---- relaxed load update (a separate variant; the default everywhere else is the rule) -------
+def _run_relaxed(dev, hb, wb, bias, loads0, k, c, eps, tfix, G, B):
+    import torch
+
+    from paper_2510_03293_b200 import laser
+
+    T, d = hb.shape
+    E = wb.shape[0]
+    p = laser.make_params(T, d, E, k, c, eps, tfix, 1, B, update_granularity=G)
+    loads = torch.from_numpy(loads0.copy()).to(dev)
+    bins = torch.zeros(B, dtype=torch.int32, device=dev)
+    r = laser.route(to_dev_bf16(hb, dev), to_dev_bf16(wb, dev), torch.from_numpy(bias).to(dev),
+                    loads, p, bin_loads=bins, want_logits=True)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    return r, loads, bins
+
+
+@pytest.mark.parametrize("router", ["tile", "splitk"])
+@pytest.mark.parametrize("T,d,E,k,c,eps,tfix", [
+    (1500, 256, 8, 2, 4, 0.7, 0.4),      # E <= 32 path
+    (1500, 256, 64, 6, 10, 0.5, 0.4),    # shared-memory masks
+    (700, 128, 256, 8, 40, 0.30, 0.10),  # one-warp scan (candidate sets wider than a warp)
+])
+@pytest.mark.parametrize("G", [0, 32, 96, 256, 1024])
+def test_relaxed_granularity_matches_its_oracle(cuda_device, monkeypatch, router, T, d, E, k, c,
+                                                eps, tfix, G):
+    monkeypatch.setenv("LASER_ROUTER", router)
+    hb, wb, bias = layer(T, d, E, seed=400 + E + G, sigma=0.05)
+    loads0 = np.random.default_rng(G + E).integers(0, 4, E).astype(np.int32)
+    B = 4
+    r, loads, bins = _run_relaxed(cuda_device, hb, wb, bias, loads0, k, c, eps, tfix, G, B)
+    x = r.logits.cpu().numpy()
+    ref = oracle.route_full(hb, wb, bias, loads0, synth.default_expert_to_bin(E, B),
+                            np.zeros(B, np.int32), k, c, eps, tfix, True, x=x, granularity=G)
+    assert np.array_equal(r.expert_ids.cpu().numpy(), ref["expert_ids"])
+    assert np.array_equal(r.offsets.cpu().numpy(), ref["offsets"])
+    assert np.array_equal(r.perm.cpu().numpy(), ref["perm"])
+    assert np.array_equal(loads.cpu().numpy(), ref["loads"])
+    assert np.array_equal(bins.cpu().numpy(), ref["bin_loads"])
+    assert np.array_equal(r.weights.cpu().numpy().view(np.uint32), ref["weights"].view(np.uint32))
+    if G in (32, 96):   # the variant really differs from the rule on these inputs
+        exact = oracle.route(x, loads0, k, c, eps, tfix, True)
+        assert not np.array_equal(exact[0], ref["expert_ids"])
