@@ -232,11 +232,25 @@ def run_gpu(args, w):
 
     L = w.layers if args.layers is None else args.layers
     data = synth.make_workload_torch(w, dev, seed=args.seed + rank, layers=L)
-    p = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize, w.n_bins)
+    p = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize, w.n_bins,
+                          update_granularity=args.granularity)
     loads = torch.zeros((L, w.E), dtype=torch.int32, device=dev)
     bins = torch.zeros((L, w.n_bins), dtype=torch.int32, device=dev)
     ws = torch.empty((laser.workspace_bytes(p) * L,), dtype=torch.uint8, device=dev)
     out = None
+    exact_ids = exact_imb = None
+    if args.granularity != 1:
+        # the rule's own result on the same inputs, to report how far the variant drifts
+        p1 = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize,
+                               w.n_bins)
+        r1 = laser.route_layers(data["hidden"], data["w_g"], data["bias"], loads, p1,
+                                bin_loads=bins, eps_high=data["eps_high"], t_fix=data["t_fix"],
+                                workspace=ws)
+        torch.cuda.synchronize()
+        exact_ids = r1.expert_ids.sort(dim=2).values.clone()
+        c1 = (r1.offsets[:, 1:] - r1.offsets[:, :-1]).double()
+        exact_imb = float((c1.max(1).values / c1.mean(1)).mean().item())
+        del r1
 
     # inputs that fit the 126 MB L2 are rotated over enough copies to exceed twice its size
     in_bytes = data["hidden"].numel() * 2
@@ -305,6 +319,9 @@ def run_gpu(args, w):
         "path": {"router_select_ms": k1, "dispatch_ms": k3, "path_gbs": path_gbs,
                  "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
         "routing": {"mean_imbalance_max_over_mean": imb, "status_word": status},
+        "variant": ("the method's rule: loads updated after every token" if args.granularity == 1
+                    else "RELAXED, not the method's rule: loads seen refreshed every %s tokens"
+                    % (args.granularity or "call (snapshot)")),
         "gpu_launches": launches_per_step(w, L) * args.steps,
         "clocks": clocks,
     }
@@ -314,6 +331,11 @@ def run_gpu(args, w):
         result["e2e"] = e2e_host(args, w, L, data, p, laser, torch, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(args, w, L, data, np)
+    if exact_ids is not None:
+        same = (out.expert_ids.sort(dim=2).values == exact_ids).all(dim=2)
+        result["drift_from_the_rule"] = {
+            "tokens_with_a_different_expert_set": float(1.0 - same.double().mean().item()),
+            "mean_imbalance_of_the_rule": exact_imb, "mean_imbalance_of_this_variant": imb}
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -498,6 +520,10 @@ def main():
                     help="override eps_high of every layer (0 = vanilla top-k, 2 = always expand)")
     ap.add_argument("--t-fix", type=float, default=None, help="override t_fix of every layer")
     ap.add_argument("--c", type=int, default=None, help="override the trimming size c")
+    ap.add_argument("--granularity", type=int, default=1,
+                    help="load-update granularity: 1 = the method's rule (default); 0 or a "
+                         "multiple of 32 = the RELAXED variant, reported as such with its drift "
+                         "from the rule")
     args = ap.parse_args()
 
     from paper_2510_03293_b200 import synth
