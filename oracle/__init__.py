@@ -51,6 +51,11 @@ def lib() -> ctypes.CDLL:
         L.lo_route.restype = i32
         L.lo_route_relaxed.argtypes = [vp, i32, i32, i32, i32, f32, f32, i32, i32, vp, vp, vp, vp]
         L.lo_route_relaxed.restype = i32
+        L.lo_philox4x32_10.argtypes = [vp, vp, vp]
+        L.lo_philox4x32_10.restype = None
+        L.lo_route_random.argtypes = [vp, i32, i32, i32, i32, f32, f32, i32, ctypes.c_uint64, i32,
+                                      vp, vp, vp, vp, vp]
+        L.lo_route_random.restype = i32
         L.lo_topk.argtypes = [vp, i32, i32, i32, vp]
         L.lo_topk.restype = None
         L.lo_dispatch.argtypes = [vp, i32, i32, i32, vp, vp]
@@ -131,6 +136,34 @@ def route_relaxed(x: np.ndarray, loads: np.ndarray, k: int, c: int, eps_high: fl
     if rc != 0:
         raise ValueError("lo_route_relaxed rejected its arguments")
     return ids, w, L, cs
+
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    """Four 32-bit words of Philox4x32-10 for a 4-word counter and a 2-word key."""
+    ctr = _c(counter, np.uint32)
+    ky = _c(key, np.uint32)
+    out = np.empty(4, np.uint32)
+    lib().lo_philox4x32_10(_p(ctr), _p(ky), _p(out))
+    return out
+
+
+def route_random(x: np.ndarray, loads: np.ndarray, k: int, c: int, eps_high: float, t_fix: float,
+                 seed: int, layer: int = 0, renormalize: bool = True):
+    """Routing with RANDOM trimming (the pool is sampled down to c* candidates with Philox).
+    Returns (expert_ids, weights, loads_out, cstar, cand [T,c] with -1 for unused)."""
+    x = _c(x, np.float32)
+    T, E = x.shape
+    L = _c(loads, np.int32).copy()
+    ids = np.empty((T, k), np.int32)
+    w = np.empty((T, k), np.float32)
+    cs = np.empty((T,), np.int32)
+    cand = np.empty((T, c), np.int32)
+    rc = lib().lo_route_random(_p(x), T, E, k, c, eps_high, t_fix, int(bool(renormalize)),
+                               ctypes.c_uint64(int(seed)), int(layer), _p(L), _p(ids), _p(w), _p(cs),
+                               _p(cand))
+    if rc != 0:
+        raise ValueError("lo_route_random rejected its arguments")
+    return ids, w, L, cs, cand
 
 
 def topk(x: np.ndarray, k: int) -> np.ndarray:

@@ -251,6 +251,115 @@ int32_t lo_route_relaxed(const float* x, int32_t T, int32_t E, int32_t k, int32_
 }
 
 /*
+ * Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+ * SC 2011): a counter-based generator, out = f(counter[4], key[2]).  Ten rounds of
+ *   hi0:lo0 = M0 * c0, hi1:lo1 = M1 * c2;  (c0,c1,c2,c3) <- (hi1^c1^k0, lo1, hi0^c3^k1, lo0)
+ * with the key bumped by the Weyl constants between rounds.
+ */
+void lo_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += W0; k1 += W1;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/*
+ * LASER routing with RANDOM trimming (Algorithm 1, mode RANDOM: "sample c* indices uniformly
+ * from T", without replacement; Final assignment in The Method).  The paper fixes neither a
+ * generator nor a sampling procedure; this library's convention:
+ *   pool    P = (pi(0), ..., pi(m-1)),  m = max(k, #{i : s_i >= t_fix * s_pi(0)})  -- the
+ *           thresholded set united with the top-k is a prefix of the score ranking
+ *   c*      = min(c, m);  if c* == m nothing is drawn and Cand = P
+ *   draws   u_0, u_1, ...: 32-bit words of Philox4x32-10 with key = (seed low, seed high) and
+ *           counter = (token index, layer, block, 0); draw i is word i % 4 of block i / 4
+ *   sample  partial Fisher-Yates: for i = 0 .. c*-1:  j = i + u_i mod (m - i);  swap P[i], P[j]
+ *   Cand    = {P[0..c*-1]}, listed in score-rank order; then, as in lo_route, the k
+ *           candidates with the smallest (load, score rank), loads updated after every token.
+ * Unlike TOP trimming the k best need not survive the sampling.  cstar[t] = 0 on the top-k
+ * branch, else c*.  cand_out, if not NULL, receives the c* sampled experts of every token in
+ * score-rank order ([T, c], unused entries -1).
+ */
+int32_t lo_route_random(const float* x, int32_t T, int32_t E, int32_t k, int32_t c,
+                        float eps_high, float t_fix, int32_t renormalize, uint64_t seed,
+                        int32_t layer, int32_t* loads, int32_t* ids, float* weights,
+                        int32_t* cstar, int32_t* cand_out) {
+    if (T < 0 || E < 1 || k < 1 || k > c || c > E) return -1;
+    float* s = (float*)malloc(sizeof(float) * (size_t)E);
+    ranked_t* pi = (ranked_t*)malloc(sizeof(ranked_t) * (size_t)E);
+    int32_t* P = (int32_t*)malloc(sizeof(int32_t) * (size_t)E);     /* rank positions */
+    int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)E);
+    if (!s || !pi || !P || !cand) { free(s); free(pi); free(P); free(cand); return -1; }
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+
+    for (int32_t t = 0; t < T; ++t) {
+        const float* xt = x + (int64_t)t * E;
+        lo_softmax(xt, E, s);
+        for (int32_t e = 0; e < E; ++e) { pi[e].x = xt[e]; pi[e].e = e; }
+        qsort(pi, (size_t)E, sizeof(ranked_t), rank_cmp);
+        float Mk = s[pi[0].e];
+        for (int32_t j = 1; j < k; ++j) Mk = Mk + s[pi[j].e];
+        int32_t* A = ids + (int64_t)t * k;
+        if (cand_out) for (int32_t j = 0; j < c; ++j) cand_out[(int64_t)t * c + j] = -1;
+        if (Mk >= eps_high) {
+            for (int32_t j = 0; j < k; ++j) A[j] = pi[j].e;
+            if (cstar) cstar[t] = 0;
+        } else {
+            float thr = t_fix * s[pi[0].e];
+            int32_t m = 0;
+            for (int32_t e = 0; e < E; ++e) if (s[e] >= thr) ++m;
+            if (m < k) m = k;
+            int32_t cs = c < m ? c : m;
+            for (int32_t i = 0; i < m; ++i) P[i] = i;
+            if (cs < m) {
+                uint32_t blk[4];
+                for (int32_t i = 0; i < cs; ++i) {
+                    if ((i & 3) == 0) {
+                        const uint32_t ctr[4] = {(uint32_t)t, (uint32_t)layer, (uint32_t)(i >> 2), 0u};
+                        lo_philox4x32_10(ctr, key, blk);
+                    }
+                    int32_t j = i + (int32_t)(blk[i & 3] % (uint32_t)(m - i));
+                    int32_t tmp = P[i]; P[i] = P[j]; P[j] = tmp;
+                }
+            }
+            /* the sample in score-rank order */
+            for (int32_t i = 1; i < cs; ++i) {
+                int32_t v = P[i], pos = i;
+                while (pos > 0 && P[pos - 1] > v) { P[pos] = P[pos - 1]; --pos; }
+                P[pos] = v;
+            }
+            if (cand_out) for (int32_t j = 0; j < cs; ++j) cand_out[(int64_t)t * c + j] = pi[P[j]].e;
+            /* by (load, position in the sample), first k */
+            for (int32_t j = 0; j < cs; ++j) {
+                int32_t pos = j;
+                while (pos > 0 && loads[pi[P[cand[pos - 1]]].e] > loads[pi[P[j]].e]) {
+                    cand[pos] = cand[pos - 1];
+                    --pos;
+                }
+                cand[pos] = j;
+            }
+            for (int32_t j = 0; j < k; ++j) A[j] = pi[P[cand[j]]].e;
+            if (cstar) cstar[t] = cs;
+        }
+        float* w = weights + (int64_t)t * k;
+        for (int32_t j = 0; j < k; ++j) w[j] = s[A[j]];
+        if (renormalize) {
+            float sum = w[0];
+            for (int32_t j = 1; j < k; ++j) sum = sum + w[j];
+            for (int32_t j = 0; j < k; ++j) w[j] = w[j] / sum;
+        }
+        for (int32_t j = 0; j < k; ++j) loads[A[j]] += 1;
+    }
+    free(s); free(pi); free(P); free(cand);
+    return 0;
+}
+
+/*
  * Vanilla top-k routing (Introduction: "selects the k experts with the highest scores";
  * the Baselines paragraph).  Written independently of lo_route: k rounds of argmax over
  * the logits with already-taken experts masked out; ties go to the lower index.

@@ -332,3 +332,91 @@ def test_relaxed_matches_a_python_restatement():
         for e in A:
             loads[e] += 1
     assert loads == L.tolist()
+
+
+# ---- RANDOM trimming ---------------------------------------------------------------------
+def test_philox_known_answers():
+    # known-answer vectors of Philox4x32-10 from the generator's reference distribution
+    # (counter and key all zero; all ones; the digits of pi)
+    kat = [
+        ([0, 0, 0, 0], [0, 0], [0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8]),
+        ([0xffffffff] * 4, [0xffffffff] * 2, [0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd]),
+        ([0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344], [0xa4093822, 0x299f31d0],
+         [0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1]),
+    ]
+    for ctr, key, want in kat:
+        assert oracle.philox4x32_10(ctr, key).tolist() == want
+
+
+def test_random_trimming_without_anything_to_trim_is_top_trimming():
+    x = _rand_logits(400, 8, 11, 0.5)
+    L0 = np.arange(8, dtype=np.int32)
+    a = oracle.route(x, L0, 2, 8, 0.7, 0.5)            # c = E: the pool is never trimmed
+    b = oracle.route_random(x, L0, 2, 8, 0.7, 0.5, seed=99)
+    for u, v in zip(a, b[:4]):
+        assert np.array_equal(u, v)
+
+
+def test_random_sample_is_a_subset_of_the_pool_of_the_right_size():
+    x = _rand_logits(500, 16, 12, 0.3)
+    k, c, eps, tf = 2, 5, 0.9, 0.5
+    ids, _, L, cs, cand = oracle.route_random(x, np.zeros(16, np.int32), k, c, eps, tf, seed=5)
+    S = oracle.softmax(x)
+    assert int(L.sum()) == 500 * k
+    for t in range(500):
+        if cs[t] == 0:
+            continue
+        order = lit.score_order(S[t], x[t])
+        m = max(k, int((S[t] >= np.float32(np.float32(tf) * S[t][order[0]])).sum()))
+        pool = set(order[:m])
+        got = [e for e in cand[t] if e >= 0]
+        assert len(got) == cs[t] == min(c, m) and len(set(got)) == len(got)
+        assert set(got) <= pool and set(ids[t]) <= set(got)
+        # listed in score-rank order; chosen = the k least loaded of the sample is checked
+        # by the brute-force selector on the loads the token saw (recomputed below)
+        assert [order.index(e) for e in got] == sorted(order.index(e) for e in got)
+
+
+def test_random_sampling_is_uniform_over_the_pool():
+    # equal logits: the pool is all 16 experts, c = 4 of them are drawn; over 4000 tokens every
+    # expert must enter the sample about 4000 * 4 / 16 = 1000 times
+    x = np.zeros((4000, 16), np.float32)
+    _, _, _, cs, cand = oracle.route_random(x, np.zeros(16, np.int32), 2, 4, 2.0, 1.0, seed=2024)
+    assert np.all(cs == 4)
+    counts = np.bincount(cand[cand >= 0], minlength=16)
+    assert counts.sum() == 16000 and counts.min() > 880 and counts.max() < 1120
+    # and different seeds draw different samples
+    cand2 = oracle.route_random(x, np.zeros(16, np.int32), 2, 4, 2.0, 1.0, seed=2025)[4]
+    assert not np.array_equal(cand, cand2)
+
+
+def test_random_trimming_python_restatement():
+    x = _rand_logits(120, 8, 13, 0.3)
+    k, c, eps, tf, seed, layer = 2, 3, 0.9, 0.3, 0x1234567890abcdef, 4
+    ids, _, L, cs, cand = oracle.route_random(x, np.zeros(8, np.int32), k, c, eps, tf, seed, layer)
+    S = oracle.softmax(x)
+    loads = [0] * 8
+    key = [seed & 0xffffffff, seed >> 32]
+    for t in range(120):
+        order = lit.score_order(S[t], x[t])
+        Mk = np.float32(S[t][order[0]])
+        for j in range(1, k):
+            Mk = np.float32(Mk + S[t][order[j]])
+        if Mk >= np.float32(eps):
+            A = order[:k]
+        else:
+            thr = np.float32(np.float32(tf) * S[t][order[0]])
+            m = max(k, int((S[t] >= thr).sum()))
+            P = list(range(m))
+            cs_t = min(c, m)
+            if cs_t < m:
+                for i in range(cs_t):
+                    u = int(oracle.philox4x32_10([t, layer, i // 4, 0], key)[i % 4])
+                    j = i + u % (m - i)
+                    P[i], P[j] = P[j], P[i]
+            sample = sorted(P[:cs_t])
+            A = lit.brute_force_token([order[r] for r in sample], loads, k)
+        assert list(ids[t]) == list(A), t
+        for e in A:
+            loads[e] += 1
+    assert loads == L.tolist()
