@@ -233,7 +233,9 @@ def run_gpu(args, w):
     L = w.layers if args.layers is None else args.layers
     data = synth.make_workload_torch(w, dev, seed=args.seed + rank, layers=L)
     p = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize, w.n_bins,
-                          update_granularity=args.granularity)
+                          update_granularity=args.granularity,
+                          trim_mode=0 if args.random_trim is None else 1,
+                          seed=args.random_trim or 0)
     loads = torch.zeros((L, w.E), dtype=torch.int32, device=dev)
     bins = torch.zeros((L, w.n_bins), dtype=torch.int32, device=dev)
     ws = torch.empty((laser.workspace_bytes(p) * L,), dtype=torch.uint8, device=dev)
@@ -319,6 +321,8 @@ def run_gpu(args, w):
         "path": {"router_select_ms": k1, "dispatch_ms": k3, "path_gbs": path_gbs,
                  "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
         "routing": {"mean_imbalance_max_over_mean": imb, "status_word": status},
+        "trimming": "TOP" if args.random_trim is None else "RANDOM (Philox4x32-10, seed %d)" %
+                    args.random_trim,
         "variant": ("the method's rule: loads updated after every token" if args.granularity == 1
                     else "RELAXED, not the method's rule: loads seen refreshed every %s tokens"
                     % (args.granularity or "call (snapshot)")),
@@ -520,6 +524,9 @@ def main():
                     help="override eps_high of every layer (0 = vanilla top-k, 2 = always expand)")
     ap.add_argument("--t-fix", type=float, default=None, help="override t_fix of every layer")
     ap.add_argument("--c", type=int, default=None, help="override the trimming size c")
+    ap.add_argument("--random-trim", type=int, default=None, metavar="SEED",
+                    help="RANDOM trimming (Algorithm 1's second mode) with this generator seed "
+                         "instead of TOP trimming")
     ap.add_argument("--granularity", type=int, default=1,
                     help="load-update granularity: 1 = the method's rule (default); 0 or a "
                          "multiple of 32 = the RELAXED variant, reported as such with its drift "

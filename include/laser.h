@@ -72,8 +72,13 @@ enum { LASER_MAX_EXPERTS = 256 };
  *                every token, a value above 1 expands every token.
  *   t_fix        pool threshold relative to the best score; paper's domain (0,1], 0 allowed
  *                (pool = the c best).  eps_high > 1, t_fix = 0, c = E is load-only routing.
- *   trim_mode    0 = TOP (keep the c best).  1 = RANDOM is not implemented
- *                (LASER_ERR_UNSUPPORTED).
+ *   trim_mode    0 = TOP (keep the c best of the pool).  1 = RANDOM (Algorithm 1's second mode):
+ *                the pool, i.e. the first m = max(k, #{s_i >= t_fix * s_max}) experts of the
+ *                score ranking, is sampled down to c* = min(c, m) candidates without
+ *                replacement.  The paper names no generator; this library draws with
+ *                Philox4x32-10, key = seed, counter = (token index, layer index in the call,
+ *                block, 0), by a partial Fisher-Yates shuffle (j = i + u_i mod (m - i)), so a
+ *                call is reproducible from (seed, inputs).  Not a tuned path.
  *   update_granularity  1 = the loads a token sees include every earlier token (the method's
  *                rule as this library reads it, and the default of every helper).
  *                0 or a multiple of 32 = RELAXED variant, not the rule and never chosen for
@@ -95,7 +100,7 @@ typedef struct laser_params {
   int32_t renormalize;
   int32_t n_bins;
   int64_t ld_hidden, ld_w;
-  uint64_t seed; /* reserved for RANDOM trimming */
+  uint64_t seed; /* RANDOM trimming: generator key */
 } laser_params;
 
 /* Library version, major*10000 + minor*100 + patch. */

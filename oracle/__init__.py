@@ -193,13 +193,19 @@ def bins(counts: np.ndarray, expert_to_bin: np.ndarray, bin_loads: np.ndarray) -
 
 
 def route_full(hidden_bits, wg_bits, bias, loads, expert_to_bin, bin_loads,
-               k, c, eps_high, t_fix, renormalize=True, x=None, granularity=1):
+               k, c, eps_high, t_fix, renormalize=True, x=None, granularity=1,
+               random_seed=None, layer=0):
     """Whole path: logits (unless given) -> routing -> dispatch -> bins.  Dict of arrays.
-    ``granularity != 1`` selects the relaxed load update of ``route_relaxed``."""
+    ``granularity != 1`` selects the relaxed load update of ``route_relaxed``; ``random_seed``
+    selects RANDOM trimming (``route_random``) for layer index ``layer``."""
     if x is None:
         x = logits(hidden_bits, wg_bits, bias)
     E = x.shape[1]
-    if granularity == 1:
+    if random_seed is not None:
+        assert granularity == 1
+        ids, w, L, cs, _ = route_random(x, loads, k, c, eps_high, t_fix, random_seed, layer,
+                                        renormalize)
+    elif granularity == 1:
         ids, w, L, cs = route(x, loads, k, c, eps_high, t_fix, renormalize)
     else:
         ids, w, L, cs = route_relaxed(x, loads, k, c, eps_high, t_fix, granularity, renormalize)

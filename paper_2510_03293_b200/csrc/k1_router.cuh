@@ -85,6 +85,116 @@ __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int 
   }
 }
 
+// ---- RANDOM trimming (Algorithm 1, mode RANDOM) ---------------------------------------------
+// Philox4x32-10 (Salmon et al., SC 2011): ten rounds of
+//   (c0,c1,c2,c3) <- (hi(M1*c2)^c1^k0, lo(M1*c2), hi(M0*c0)^c3^k1, lo(M0*c0)),
+// the key advancing by the Weyl constants between rounds.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t n0 = __umulhi(M1, c2) ^ c1 ^ k0, n1 = M1 * c2;
+    const uint32_t n2 = __umulhi(M0, c0) ^ c3 ^ k1, n3 = M0 * c0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Per-token epilogue with RANDOM trimming, one thread on a row of logits in shared memory.
+// Softmax, ranking and the top-k mass test are those of token_epilogue.  On the expanded branch
+//   pool  = ranking prefix of length m = max(k, #{i : s_i >= t_fix * s_pi(0)}) over all E,
+//   c*    = min(c, m); if c* < m a partial Fisher-Yates shuffle draws the sample:
+//           for i < c*:  j = i + u_i mod (m - i), swap  (u_i = word i % 4 of the Philox block
+//           with key = seed and counter = (token, layer, i / 4, 0)),
+//   the record lists the c* sampled experts in score-rank order.
+// Not a fast path: it ranks up to E experts round by round and keeps two byte arrays in local
+// memory.
+__device__ __noinline__ void token_epilogue_random(const float* row, int E, int k, int c,
+                                                   float eps_high, float t_fix, int renorm,
+                                                   unsigned long long seed, int layer, long long t,
+                                                   uint16_t* cstar, uint8_t* cand_ids,
+                                                   float* cand_scores, int32_t* expert_ids,
+                                                   float* weights) {
+  float xmax = row[0];
+  for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, row[i]);
+  float a[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) a[j] = 0.0f;
+  for (int i0 = 0; i0 < E; i0 += 8) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (i0 + j < E) a[j] = __fadd_rn(a[j], exp32(__fsub_rn(row[i0 + j], xmax)));
+  }
+  const float Z = __fadd_rn(__fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3])),
+                            __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7])));
+  const float thr = __fmul_rn(t_fix, __fdiv_rn(exp32(0.0f), Z));   // s of the best expert
+  int m = 0;
+  for (int i = 0; i < E; ++i)
+    if (__fdiv_rn(exp32(__fsub_rn(row[i], xmax)), Z) >= thr) ++m;
+  if (m < k) m = k;
+
+  uint8_t R[kMaxExperts];   // R[r]: expert of rank r
+  uint8_t P[kMaxExperts];   // rank positions, shuffled
+  float prev_x = __int_as_float(0x7f800000);  // +inf
+  int prev_i = -1;
+  float Mk = 0.0f;
+  int need = k;
+  for (int r = 0; r < need; ++r) {
+    float bx = 0.0f;
+    int bi = -1;
+    for (int i = 0; i < E; ++i) {
+      const float xi = row[i];
+      const bool after_prev = (xi < prev_x) || (xi == prev_x && i > prev_i);
+      if (after_prev && (bi < 0 || xi > bx)) { bx = xi; bi = i; }
+    }
+    R[r] = (uint8_t)bi;
+    if (r < k) {
+      const float s = __fdiv_rn(exp32(__fsub_rn(bx, xmax)), Z);
+      Mk = r == 0 ? s : __fadd_rn(Mk, s);
+      expert_ids[r] = bi;
+      weights[r] = s;
+      cand_ids[r] = (uint8_t)bi;   // the top-k branch's record: the selection and the dispatch
+      cand_scores[r] = s;          // read the k best from here (overwritten by a sample)
+      if (r == k - 1 && !(Mk >= eps_high)) need = m;   // expanded: rank the whole pool
+    }
+    prev_x = bx;
+    prev_i = bi;
+  }
+  if (Mk >= eps_high) {
+    *cstar = 0;
+    if (renorm)
+      for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
+    return;
+  }
+  const int cs = c < m ? c : m;
+  for (int i = 0; i < m; ++i) P[i] = (uint8_t)i;
+  if (cs < m) {
+    uint32_t blk[4];
+    for (int i = 0; i < cs; ++i) {
+      if ((i & 3) == 0)
+        philox4x32_10((uint32_t)t, (uint32_t)layer, (uint32_t)(i >> 2), 0u, (uint32_t)seed,
+                      (uint32_t)(seed >> 32), blk);
+      const uint32_t u = (i & 3) == 0 ? blk[0] : ((i & 3) == 1 ? blk[1] : ((i & 3) == 2 ? blk[2] : blk[3]));
+      const int j = i + (int)(u % (uint32_t)(m - i));
+      const uint8_t tmp = P[i]; P[i] = P[j]; P[j] = tmp;
+    }
+  }
+  for (int i = 1; i < cs; ++i) {   // the sample in score-rank order
+    const uint8_t v = P[i];
+    int pos = i;
+    while (pos > 0 && P[pos - 1] > v) { P[pos] = P[pos - 1]; --pos; }
+    P[pos] = v;
+  }
+  for (int j = 0; j < cs; ++j) {
+    const int e = R[P[j]];
+    cand_ids[j] = (uint8_t)e;
+    cand_scores[j] = __fdiv_rn(exp32(__fsub_rn(row[e], xmax)), Z);
+  }
+  *cstar = (uint16_t)cs;
+}
+
 // ---- score epilogue with sorting networks (one thread per token) ---------------------------
 // Descending bitonic sort of N (power of two) registers.
 template <int N>
@@ -503,11 +613,16 @@ __device__ __forceinline__ void group_epilogue(const RouteArgs& A, int layer, lo
   unsigned char* ws = A.ws + (size_t)(A.layer0 + layer) * A.ws_ls;
   const int k = A.k, c = A.c;
   const size_t lt = (size_t)(A.layer0 + layer) * A.T + t;
-  token_epilogue(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
-                 reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
-                 ws + A.lay.cand_ids + (size_t)t * c,
-                 reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
-                 A.expert_ids + lt * k, A.weights + lt * k);
+  uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
+  uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
+  float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
+  if (A.trim_random)
+    token_epilogue_random(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer],
+                          A.renorm, A.seed, A.layer0 + layer, t, cs_p, ids_p, sc_p,
+                          A.expert_ids + lt * k, A.weights + lt * k);
+  else
+    token_epilogue(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
+                   cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k);
 }
 
 
@@ -630,7 +745,20 @@ __device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int laye
       out[idx] = tile[r * LDS + e];
     }
   }
-  if (warp < 4) {
+  if (A.trim_random) {
+    const long long t = tok0 + tid;
+    if (tid < 16 && t < T) {
+      unsigned char* ws = A.ws + (size_t)abs_layer * A.ws_ls;
+      const int k = A.k, c = A.c;
+      const size_t lt = (size_t)abs_layer * T + t;
+      token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer],
+                            A.renorm, A.seed, abs_layer, t,
+                            reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
+                            ws + A.lay.cand_ids + (size_t)t * c,
+                            reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
+                            A.expert_ids + lt * k, A.weights + lt * k);
+    }
+  } else if (warp < 4) {
     const int r = warp * 4 + (lane >> 3);
     const long long t = tok0 + r;
     const bool write = t < T;

@@ -270,7 +270,11 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
         uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
         uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
         float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
-        if (c <= CL)
+        if (A.trim_random)
+          token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
+                                A.t_fix[layer], A.renorm, A.seed, abs_layer, t, cs_p, ids_p, sc_p,
+                                A.expert_ids + lt * k, A.weights + lt * k);
+        else if (c <= CL)
           token_epilogue_sorted<N, CL>(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
                                        A.t_fix[layer], A.renorm, cs_p, ids_p, sc_p,
                                        A.expert_ids + lt * k, A.weights + lt * k);
@@ -312,10 +316,22 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
           out[idx] = tile[r * LDS + e];
         }
       }
+      if (A.trim_random) {   // one thread per token of this pass
+        const long long t = tok0 + tid;
+        if (tid < ROWS && t < T) {
+          const size_t lt = (size_t)abs_layer * T + t;
+          token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
+                                A.t_fix[layer], A.renorm, A.seed, abs_layer, t,
+                                reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
+                                ws + A.lay.cand_ids + (size_t)t * c,
+                                reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
+                                A.expert_ids + lt * k, A.weights + lt * k);
+        }
+      }
       // groups of 8 lanes score one token each, 4 tokens per warp at a time
       const int g = lane >> 3, j = lane & 7;
 #pragma unroll 1
-      for (int it = 0; it < ROWS / 32; ++it) {
+      for (int it = 0; it < (A.trim_random ? 0 : ROWS / 32); ++it) {
         const int r = warp * (ROWS / 8) + it * 4 + g;
         const long long t = tok0 + r;
         const bool write = t < T;

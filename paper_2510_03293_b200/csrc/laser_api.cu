@@ -22,8 +22,7 @@ int validate_params(const laser_params* p) {
   if (p->d % 8 != 0) return LASER_ERR_INVALID_ARG;
   if (!(p->eps_high >= 0.0f) || !(p->t_fix >= 0.0f) || !(p->t_fix <= 1.0f))
     return LASER_ERR_INVALID_ARG;
-  if (p->trim_mode == 1) return LASER_ERR_UNSUPPORTED;
-  if (p->trim_mode != 0) return LASER_ERR_INVALID_ARG;
+  if (p->trim_mode != 0 && p->trim_mode != 1) return LASER_ERR_INVALID_ARG;
   if (p->update_granularity < 0) return LASER_ERR_INVALID_ARG;
   if (p->update_granularity != 1 && p->update_granularity % 32 != 0) return LASER_ERR_UNSUPPORTED;
   if (p->n_bins < 1) return LASER_ERR_INVALID_ARG;
@@ -298,6 +297,8 @@ extern "C" int laser_route_layers_profiled(
   a.T = p->T; a.d = p->d; a.E = p->E; a.k = p->k; a.c = p->c;
   a.n_bins = p->n_bins; a.renorm = p->renormalize ? 1 : 0;
   a.G = p->update_granularity;
+  a.trim_random = p->trim_mode == 1 ? 1 : 0;
+  a.seed = p->seed;
   a.ld_h = p->ld_hidden; a.ld_w = p->ld_w;
 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

@@ -55,6 +55,8 @@ struct RouteArgs {
   unsigned char* ws;       size_t ws_ls;          // bytes
   WorkspaceLayout lay;
   int T, d, E, k, c, n_bins, renorm;
+  int trim_random;         // 1 = RANDOM trimming of the pool (Philox draws), 0 = TOP
+  unsigned long long seed; // RANDOM trimming: generator key
   int G;                   // load-update granularity: 1 = after every token (the rule);
                            // 0 or a multiple of 32 = relaxed variant (loads seen refreshed
                            // every G tokens, 0 = once per call)

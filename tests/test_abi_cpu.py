@@ -48,7 +48,6 @@ def good(**over):
     (dict(n_bins=0), laser.ERR_INVALID_ARG),
     (dict(ld_hidden=128), laser.ERR_INVALID_ARG),
     (dict(ld_hidden=260), laser.ERR_MISALIGNED),
-    (dict(trim_mode=1), laser.ERR_UNSUPPORTED),
     (dict(trim_mode=7), laser.ERR_INVALID_ARG),
     (dict(update_granularity=7), laser.ERR_UNSUPPORTED),
     (dict(update_granularity=-32), laser.ERR_INVALID_ARG),

@@ -325,3 +325,49 @@ def test_relaxed_granularity_matches_its_oracle(cuda_device, monkeypatch, router
     if G in (32, 96):   # the variant really differs from the rule on these inputs
         exact = oracle.route(x, loads0, k, c, eps, tfix, True)
         assert not np.array_equal(exact[0], ref["expert_ids"])
+
+
+# ---- RANDOM trimming -------------------------------------------------------------------
+@pytest.mark.parametrize("router", ["tile", "splitk"])
+@pytest.mark.parametrize("T,d,E,k,c,eps,tfix", [
+    (900, 256, 8, 2, 3, 0.8, 0.3),       # warp-level / split-K routers
+    (900, 256, 64, 6, 8, 0.6, 0.3),      # tensor-memory router, 64 columns
+    (600, 128, 100, 5, 12, 0.5, 0.2),    # 128 columns
+    (500, 128, 256, 8, 16, 0.3, 0.3),    # 256 columns (two-pass epilogue)
+])
+def test_random_trimming_matches_its_oracle(cuda_device, monkeypatch, router, T, d, E, k, c, eps,
+                                            tfix):
+    import torch
+
+    from paper_2510_03293_b200 import laser
+
+    monkeypatch.setenv("LASER_ROUTER", router)
+    dev = cuda_device
+    Lr, B, seed = 2, 4, 0xC0FFEE1234
+    layers = [layer(T, d, E, seed=500 + l + E, sigma=0.08) for l in range(Lr)]
+    hb = np.stack([x[0] for x in layers]); wb = np.stack([x[1] for x in layers])
+    bias = np.stack([x[2] for x in layers])
+    p = laser.make_params(T, d, E, k, c, eps, tfix, 1, B, trim_mode=1, seed=seed)
+    loads = torch.zeros((Lr, E), dtype=torch.int32, device=dev)
+    bins = torch.zeros((Lr, B), dtype=torch.int32, device=dev)
+    r = laser.route_layers(to_dev_bf16(hb, dev), to_dev_bf16(wb, dev),
+                           torch.from_numpy(bias).to(dev), loads, p, bin_loads=bins,
+                           want_logits=True)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    trimmed = 0
+    for l in range(Lr):
+        x = r.logits[l].cpu().numpy()
+        ref = oracle.route_full(hb[l], wb[l], bias[l], np.zeros(E, np.int32),
+                                synth.default_expert_to_bin(E, B), np.zeros(B, np.int32), k, c,
+                                eps, tfix, True, x=x, random_seed=seed, layer=l)
+        assert np.array_equal(r.expert_ids[l].cpu().numpy(), ref["expert_ids"]), l
+        assert np.array_equal(r.offsets[l].cpu().numpy(), ref["offsets"])
+        assert np.array_equal(r.perm[l].cpu().numpy(), ref["perm"])
+        assert np.array_equal(loads[l].cpu().numpy(), ref["loads"])
+        assert np.array_equal(bins[l].cpu().numpy(), ref["bin_loads"])
+        assert np.array_equal(r.weights[l].cpu().numpy().view(np.uint32),
+                              ref["weights"].view(np.uint32))
+        top = oracle.route(x, np.zeros(E, np.int32), k, c, eps, tfix, True)
+        trimmed += int((top[0] != ref["expert_ids"]).any(1).sum())
+    assert trimmed > 0   # the sampling really changed assignments on these inputs
