@@ -306,8 +306,8 @@ def run_gpu(args, w):
     path_gbs = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
 
     status = int(out.status.item())
-    counts = (out.offsets[:, 1:] - out.offsets[:, :-1]).double()
-    imb = float((counts.max(1).values / counts.mean(1)).mean().item())
+    I_layers, I_bins, I_agg = laser.imbalance(out.offsets, w.n_bins)
+    imb = float(I_layers.double().mean().item())
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -320,7 +320,10 @@ def run_gpu(args, w):
                      "bytes_per_launch": bytes_per_launch},
         "path": {"router_select_ms": k1, "dispatch_ms": k3, "path_gbs": path_gbs,
                  "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
-        "routing": {"mean_imbalance_max_over_mean": imb, "status_word": status},
+        "routing": {"mean_imbalance_max_over_mean": imb, "I_agg": float(I_agg[0].item()),
+                    "I_agg_bins": float(I_agg[1].item()),
+                    "MV_max_over_layers": float(I_layers.max().item()) - 1.0,
+                    "status_word": status},
         "trimming": "TOP" if args.random_trim is None else "RANDOM (Philox4x32-10, seed %d)" %
                     args.random_trim,
         "variant": ("the method's rule: loads updated after every token" if args.granularity == 1
@@ -335,6 +338,9 @@ def run_gpu(args, w):
         result["e2e"] = e2e_host(args, w, L, data, p, laser, torch, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(args, w, L, data, np)
+    if args.imbalance_batches > 0 and rank == 0:
+        result["imbalance_study"] = imbalance_study(args, w, L, data, laser, synth, torch, dev,
+                                                    loads, bins, ws)
     if exact_ids is not None:
         same = (out.expert_ids.sort(dim=2).values == exact_ids).all(dim=2)
         result["drift_from_the_rule"] = {
@@ -345,6 +351,56 @@ def run_gpu(args, w):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(result))
+
+
+def imbalance_study(args, w, L, data, laser, synth, torch, dev, loads, bins, ws):
+    """The evaluation's balance figures over several batches: I_agg (P50 and P95 over batches) and
+    MV (mean over layers and batches of I_L - 1), for the method next to its two baselines --
+    plain top-k (eps_high = 0: every token takes the top-k branch) and load-only (eps_high > 1,
+    t_fix = 0, c = E: every expert is a candidate, chosen by load alone).  Same gate weights,
+    a fresh seeded batch of hidden states each time, loads starting from zero; the figures come
+    from the imbalance kernel, the percentiles from the B values it returned."""
+    policies = {
+        "laser": dict(c=w.c, eps=data["eps_high"], tfix=data["t_fix"]),
+        "top_k": dict(c=w.c, eps=[0.0] * L, tfix=data["t_fix"]),
+        "load_only": dict(c=w.E, eps=[2.0] * L, tfix=[0.0] * L),
+    }
+    agg = {name: [] for name in policies}
+    agg_bins = {name: [] for name in policies}
+    mv = {name: [] for name in policies}
+    ws_lo = None
+    for b in range(args.imbalance_batches):
+        hidden = synth.make_workload_torch(w, dev, seed=args.seed + 7919 * (b + 1),
+                                           layers=L)["hidden"]
+        for name, pol in policies.items():
+            p = laser.make_params(w.T, w.d, w.E, w.k, pol["c"], pol["eps"][0], pol["tfix"][0],
+                                  w.renormalize, w.n_bins)
+            if pol["c"] != w.c and ws_lo is None:
+                ws_lo = torch.empty((laser.workspace_bytes(p) * L,), dtype=torch.uint8, device=dev)
+            loads.zero_(); bins.zero_()
+            r = laser.route_layers(hidden, data["w_g"], data["bias"], loads, p, bin_loads=bins,
+                                   eps_high=pol["eps"], t_fix=pol["tfix"],
+                                   workspace=ws if pol["c"] == w.c else ws_lo)
+            I, Ib, a = laser.imbalance(r.offsets, w.n_bins)
+            torch.cuda.synchronize()
+            agg[name].append(float(a[0].item()))
+            agg_bins[name].append(float(a[1].item()))
+            mv[name].append(float((I.double() - 1.0).mean().item()))
+            del r
+        del hidden
+
+    def pct(v, q):
+        s = sorted(v)
+        pos = (len(s) - 1) * q
+        lo = int(pos)
+        hi = min(lo + 1, len(s) - 1)
+        return s[lo] + (s[hi] - s[lo]) * (pos - lo)
+
+    return {"batches": args.imbalance_batches,
+            "policies": {name: {"I_agg_P50": pct(agg[name], 0.5), "I_agg_P95": pct(agg[name], 0.95),
+                                "I_agg_bins_P50": pct(agg_bins[name], 0.5),
+                                "MV_mean": sum(mv[name]) / len(mv[name])}
+                         for name in policies}}
 
 
 def run_decode(args, w):
@@ -527,6 +583,9 @@ def main():
     ap.add_argument("--random-trim", type=int, default=None, metavar="SEED",
                     help="RANDOM trimming (Algorithm 1's second mode) with this generator seed "
                          "instead of TOP trimming")
+    ap.add_argument("--imbalance-batches", type=int, default=0, metavar="B",
+                    help="after the timed run, route B more batches under the method, plain "
+                         "top-k and load-only, and report I_agg P50/P95 and MV of each")
     ap.add_argument("--granularity", type=int, default=1,
                     help="load-update granularity: 1 = the method's rule (default); 0 or a "
                          "multiple of 32 = the RELAXED variant, reported as such with its drift "

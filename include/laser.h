@@ -206,6 +206,32 @@ int laser_route_host(int32_t n_layers,
                      int32_t* status_out,
                      void* arena, size_t arena_bytes, void* cuda_stream);
 
+/*
+ * Imbalance figures of a finished call, computed on the device from its dispatch offsets
+ * [Motivation: expert imbalance I_L = max_e N_e / mean_e N_e of a layer and batch, the
+ * aggregate I_agg = sum_L w_L I_L, and the same on devices with N_g = sum_e A_{g,e} N_e for a
+ * 0/1 placement; Evaluation, Metrics: MV, read as I_L - 1].
+ *
+ *   offsets       [n_layers, E+1] int32, as written by laser_route_layers
+ *   expert_to_bin [E] int32 in [0, n_bins), or NULL for contiguous e / ceil(E / n_bins);
+ *                 ignored when placement is given
+ *   placement     [n_bins, E] fp32 row-major, or NULL: the general matrix A (A[g,e] >= 0, each
+ *                 column summing to 1; a replicated expert splits its tokens); not checked
+ *   imbalance     [n_layers] fp32 out: I_L (1 for a layer without assignments)
+ *   bin_imbalance [n_layers] fp32 out, or NULL: the same over the n_bins device bins
+ *   aggregate     [2] fp32 out, or NULL: I_agg and its bin-level counterpart (1 when
+ *                 bin_imbalance is NULL).  The paper leaves w_L open; here w_L is the layer's
+ *                 share of all assignments of the call, which is uniform for equal layers.
+ * MV of a layer is imbalance[l] - 1.  All pointers are device pointers, caller-owned.
+ * Limits: 1 <= n_layers <= 65535; 1 <= n_bins <= E without placement, <= 1024 with it.
+ * Counts are exact; bin loads and ratios are formed in fp64 and rounded once to fp32.
+ * Enqueues two small kernels on cuda_stream; returns LASER_ERR_INVALID_ARG on a bad
+ * argument and LASER_ERR_CUDA if a launch fails.
+ */
+int laser_imbalance(int32_t n_layers, int32_t E, int32_t n_bins, const int32_t* offsets,
+                    const int32_t* expert_to_bin, const float* placement, float* imbalance,
+                    float* bin_imbalance, float* aggregate, void* cuda_stream);
+
 /* Size of the scratch array built into the library for laser_route_static (4 MiB). */
 enum { LASER_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 };
 

@@ -87,6 +87,35 @@ def imbalance(counts) -> float:
     return float(counts.max() / mean) if mean > 0 else 1.0
 
 
+def imbalance_stats(counts, expert_to_bin, n_bins, placement=None):
+    """Imbalance figures of one call over several layers, in fp64 (Motivation: expert imbalance
+    I_L = max_e N_e / mean_e N_e per layer, its token-weighted aggregate I_agg = sum_L w_L I_L
+    with w_L = tokens of layer L / all tokens, and the same on device bins with
+    N_g = sum_e A[g,e] N_e; A is the 0/1 matrix of expert_to_bin unless a general placement
+    [n_bins, E] with unit column sums is given).  counts: [L, E].
+    Returns dict(I [L], MV [L] = I - 1, I_bins [L], I_agg, I_agg_bins); a layer without
+    assignments has I = 1."""
+    counts = np.asarray(counts, np.float64)
+    L, E = counts.shape
+    bins = np.zeros((L, n_bins), np.float64)
+    for e in range(E):
+        if placement is None:
+            bins[:, int(expert_to_bin[e])] += counts[:, e]
+        else:
+            for g in range(n_bins):
+                bins[:, g] += float(placement[g][e]) * counts[:, e]
+    tot = counts.sum(1)
+
+    def ratio(a):
+        mean = a.mean(1)
+        return np.where(mean > 0, a.max(1) / np.where(mean > 0, mean, 1.0), 1.0)
+
+    I, Ib = ratio(counts), ratio(bins)
+    w = tot / tot.sum() if tot.sum() > 0 else np.full(L, 1.0 / L)
+    return dict(I=I, MV=I - 1.0, I_bins=Ib, I_agg=float((w * I).sum()),
+                I_agg_bins=float((w * Ib).sum()))
+
+
 def max_violation(counts) -> float:
     """MV, read as how far the most loaded expert exceeds the average, relative to it:
     max/mean - 1 (zero for perfect balance, as the load-only baseline attains)."""

@@ -8,6 +8,7 @@
 
 #include "k12_fused.cuh"
 #include "k3_dispatch.cuh"
+#include "k4_metrics.cuh"
 
 using namespace laser;
 
@@ -232,6 +233,22 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
 }  // namespace
 
 extern "C" int laser_version(void) { return 100; }
+
+extern "C" int laser_imbalance(int32_t n_layers, int32_t E, int32_t n_bins, const int32_t* offsets,
+                               const int32_t* expert_to_bin, const float* placement,
+                               float* imbalance, float* bin_imbalance, float* aggregate,
+                               void* cuda_stream) {
+  if (n_layers < 1 || n_layers > 65535 || E < 1 || E > LASER_MAX_EXPERTS || n_bins < 1 ||
+      n_bins > (placement ? kK4MaxBins : E) || !offsets || !imbalance)
+    return LASER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  k4_imbalance<<<n_layers < 148 ? n_layers : 148, kK4Threads, 0, st>>>(
+      n_layers, E, n_bins, offsets, expert_to_bin, placement, imbalance, bin_imbalance);
+  if (aggregate)
+    k4_aggregate<<<1, kK4Threads, 0, st>>>(n_layers, E, offsets, imbalance, bin_imbalance,
+                                           aggregate);
+  return cudaGetLastError() == cudaSuccess ? LASER_OK : LASER_ERR_CUDA;
+}
 
 extern "C" const char* laser_strerror(int status) {
   switch (status) {

@@ -34,7 +34,7 @@ MAX_EXPERTS = 256
 
 EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_route",
            "laser_route_layers", "laser_route_layers_profiled", "laser_host_arena_bytes",
-           "laser_route_host", "laser_route_static")
+           "laser_route_host", "laser_route_static", "laser_imbalance")
 
 
 class LaserParams(ctypes.Structure):
@@ -70,6 +70,10 @@ _lib.laser_route_host.restype = ctypes.c_int
 _lib.laser_route_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _pp, _vp, _vp, _vp, _vp, _vp,
                                     _vp, _vp]
 _lib.laser_route_static.restype = ctypes.c_int
+
+
+_lib.laser_imbalance.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.laser_imbalance.restype = ctypes.c_int
 
 
 class LaserError(RuntimeError):
@@ -212,6 +216,26 @@ def route_static(hidden, w_g, bias, loads, p: LaserParams, out: RouteResult, *,
     if rc != OK:
         raise LaserError(rc)
     return out
+
+
+def imbalance(offsets, n_bins: int, expert_to_bin=None, placement=None, stream=None):
+    """laser_imbalance on the offsets [L, E+1] of a finished call (torch CUDA int32 tensor).
+    placement: optional [n_bins, E] fp32 matrix A (columns sum to 1), used instead of the map.
+    Returns (I [L], I_bins [L], aggregate [2] = (I_agg, bin-level I_agg)) as device tensors;
+    MV of a layer is I - 1."""
+    import torch
+
+    L, E1 = offsets.shape
+    dev = offsets.device
+    I = torch.empty((L,), dtype=torch.float32, device=dev)
+    Ib = torch.empty((L,), dtype=torch.float32, device=dev)
+    agg = torch.empty((2,), dtype=torch.float32, device=dev)
+    s = torch.cuda.current_stream(dev) if stream is None else stream
+    rc = _lib.laser_imbalance(L, E1 - 1, n_bins, _ptr(offsets), _ptr(expert_to_bin),
+                              _ptr(placement), _ptr(I), _ptr(Ib), _ptr(agg), s.cuda_stream)
+    if rc != OK:
+        raise LaserError(rc)
+    return I, Ib, agg
 
 
 def route_host(hidden, w_g, bias, loads, p: LaserParams, arena, *, expert_to_bin=None,

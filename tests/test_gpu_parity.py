@@ -371,3 +371,39 @@ def test_random_trimming_matches_its_oracle(cuda_device, monkeypatch, router, T,
         top = oracle.route(x, np.zeros(E, np.int32), k, c, eps, tfix, True)
         trimmed += int((top[0] != ref["expert_ids"]).any(1).sum())
     assert trimmed > 0   # the sampling really changed assignments on these inputs
+
+
+def test_imbalance_kernel_matches_the_fp64_figures(cuda_device):
+    import torch
+
+    from oracle import alg1_literal as lit
+    from paper_2510_03293_b200 import laser
+
+    rng = np.random.default_rng(5)
+    for Lr, E, B in [(1, 8, 4), (32, 8, 8), (27, 64, 8), (3, 256, 32), (70, 13, 5)]:
+        counts = rng.integers(0, 5000, (Lr, E)).astype(np.int64)
+        counts[0, :] = 0 if Lr > 1 else counts[0, :]          # a layer without assignments
+        e2b = rng.integers(0, B, E).astype(np.int32)
+        e2b[:B] = np.arange(B)
+        off = np.zeros((Lr, E + 1), np.int32)
+        off[:, 1:] = np.cumsum(counts, 1)
+        I, Ib, agg = laser.imbalance(torch.from_numpy(off).to(cuda_device), B,
+                                     torch.from_numpy(e2b).to(cuda_device))
+        torch.cuda.synchronize()
+        ref = lit.imbalance_stats(counts, e2b, B)
+        assert np.allclose(I.cpu().numpy(), ref["I"], rtol=2e-6, atol=0)
+        assert np.allclose(Ib.cpu().numpy(), ref["I_bins"], rtol=2e-6, atol=0)
+        assert abs(float(agg[0]) - ref["I_agg"]) <= 4e-6 * ref["I_agg"]
+        assert abs(float(agg[1]) - ref["I_agg_bins"]) <= 4e-6 * ref["I_agg_bins"]
+        # general placement: every expert split over two devices, columns summing to 1
+        A = np.zeros((B, E), np.float32)
+        f = rng.integers(1, 8, E) / 8.0
+        A[e2b, np.arange(E)] += f
+        A[(e2b + 1) % B, np.arange(E)] += 1.0 - f
+        I2, Ib2, agg2 = laser.imbalance(torch.from_numpy(off).to(cuda_device), B,
+                                        placement=torch.from_numpy(A).to(cuda_device))
+        torch.cuda.synchronize()
+        ref2 = lit.imbalance_stats(counts, None, B, A)
+        assert np.array_equal(I2.cpu().numpy(), I.cpu().numpy())
+        assert np.allclose(Ib2.cpu().numpy(), ref2["I_bins"], rtol=2e-6, atol=0)
+        assert abs(float(agg2[1]) - ref2["I_agg_bins"]) <= 4e-6 * ref2["I_agg_bins"]

@@ -420,3 +420,25 @@ def test_random_trimming_python_restatement():
         for e in A:
             loads[e] += 1
     assert loads == L.tolist()
+
+
+# ---- imbalance figures ---------------------------------------------------------------------
+def test_imbalance_stats_by_hand_and_limits():
+    counts = np.array([[4, 0, 2, 2], [1, 1, 1, 1], [0, 0, 0, 8]], np.int64)
+    st = lit.imbalance_stats(counts, [0, 0, 1, 1], 2)
+    assert st["I"].tolist() == [2.0, 1.0, 4.0] and st["MV"].tolist() == [1.0, 0.0, 3.0]
+    assert st["I_bins"].tolist() == [1.0, 1.0, 2.0]
+    # token-weighted aggregate: weights 8/20, 4/20, 8/20
+    assert abs(st["I_agg"] - (0.4 * 2 + 0.2 * 1 + 0.4 * 4)) < 1e-12
+    assert abs(st["I_agg_bins"] - (0.4 * 1 + 0.2 * 1 + 0.4 * 2)) < 1e-12
+    # a general placement: expert 3 replicated over both devices in halves
+    A = [[1, 1, 0, 0.5], [0, 0, 1, 0.5]]
+    assert lit.imbalance_stats(counts, None, 2, A)["I_bins"].tolist() == [1.25, 1.25, 1.0]
+    # the single-layer helper agrees, and I never exceeds the number of experts
+    for l in range(3):
+        assert lit.imbalance(counts[l]) == st["I"][l] <= 4
+    # load-only routing from zero loads: perfect balance, MV = 0 (the paper's baseline)
+    x = _rand_logits(800, 8, 21, 1.0)
+    L = oracle.route(x, np.zeros(8, np.int32), 2, 8, 2.0, 0.0)[2]
+    st = lit.imbalance_stats(L[None], np.arange(8) // 2, 4)
+    assert st["I"][0] == 1.0 and st["MV"][0] == 0.0 and st["I_bins"][0] == 1.0
