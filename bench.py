@@ -341,6 +341,9 @@ def run_gpu(args, w):
     if args.imbalance_batches > 0 and rank == 0:
         result["imbalance_study"] = imbalance_study(args, w, L, data, laser, synth, torch, dev,
                                                     loads, bins, ws)
+    if args.score_stats and rank == 0:
+        result["score_stats"] = score_stats_report(args, w, L, data, p, laser, torch, loads, bins,
+                                                   ws)
     if exact_ids is not None:
         same = (out.expert_ids.sort(dim=2).values == exact_ids).all(dim=2)
         result["drift_from_the_rule"] = {
@@ -401,6 +404,46 @@ def imbalance_study(args, w, L, data, laser, synth, torch, dev, loads, bins, ws)
                                 "I_agg_bins_P50": pct(agg_bins[name], 0.5),
                                 "MV_mean": sum(mv[name]) / len(mv[name])}
                          for name in policies}}
+
+
+def score_stats_report(args, w, L, data, p, laser, torch, loads, bins, ws):
+    """Gate-score statistics of the batch by layer band (thirds of the layer index): mean M_k,
+    mean entropy, regime shares, and the M_k median read off the histogram -- the figures the
+    thresholds are calibrated from.  The logits come from the routing call itself."""
+    loads.zero_(); bins.zero_()
+    r = laser.route_layers(data["hidden"], data["w_g"], data["bias"], loads, p, bin_loads=bins,
+                           eps_high=data["eps_high"], t_fix=data["t_fix"], workspace=ws,
+                           want_logits=True)
+    for _ in range(3):
+        stats, means = laser.score_stats(r.logits, w.k, 0.5, max(2, w.E // 4))
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    stats, means = laser.score_stats(r.logits, w.k, 0.5, max(2, w.E // 4))
+    t1.record()
+    torch.cuda.synchronize()
+    st, mn = stats.cpu().double(), means.cpu().double()
+    bands = {}
+    for name, lo, hi in (("early", 0, -(-L // 3)), ("middle", -(-L // 3), -(-2 * L // 3)),
+                         ("final", -(-2 * L // 3), L)):
+        if hi <= lo:
+            continue
+        s = st[lo:hi].sum(0)
+        hist = s[8:]
+        half, acc, median_bin = s[0] / 2, 0.0, 63
+        for b in range(64):
+            acc += float(hist[b])
+            if acc >= float(half):
+                median_bin = b
+                break
+        bands[name] = {"layers": [lo, hi - 1], "mean_M_k": float(mn[lo:hi, 0].mean()),
+                       "mean_entropy_nats": float(mn[lo:hi, 1].mean()),
+                       "share_single_head": float(s[3] / s[0]), "share_plateau": float(s[4] / s[0]),
+                       "share_smooth": float(s[5] / s[0]),
+                       "M_k_median_bin_of_64": median_bin}
+    return {"near_ratio": 0.5, "plateau_max": max(2, w.E // 4), "bands": bands,
+            "kernel_ms": t0.elapsed_time(t1),
+            "logits_bytes": r.logits.numel() * 4,
+            "note": "one call (memset and two kernels) on logits just written, so partly in L2"}
 
 
 def run_decode(args, w):
@@ -586,6 +629,8 @@ def main():
     ap.add_argument("--imbalance-batches", type=int, default=0, metavar="B",
                     help="after the timed run, route B more batches under the method, plain "
                          "top-k and load-only, and report I_agg P50/P95 and MV of each")
+    ap.add_argument("--score-stats", action="store_true",
+                    help="add the gate-score statistics of the batch by layer band")
     ap.add_argument("--granularity", type=int, default=1,
                     help="load-update granularity: 1 = the method's rule (default); 0 or a "
                          "multiple of 32 = the RELAXED variant, reported as such with its drift "

@@ -232,6 +232,40 @@ int laser_imbalance(int32_t n_layers, int32_t E, int32_t n_bins, const int32_t* 
                     const int32_t* expert_to_bin, const float* placement, float* imbalance,
                     float* bin_imbalance, float* aggregate, void* cuda_stream);
 
+/*
+ * Gate-score statistics per layer, from fp32 logits (e.g. logits_out of laser_route_layers on
+ * prefill batches) [Layer Variability in Gate Score Distributions: top-k mass M_k, Shannon
+ * entropy, the regimes single-head / plateau / smooth; The Method, Parameter setting: these
+ * figures guide eps_high and t_fix per layer or layer band].
+ *
+ *   logits  [n_layers, T, E] fp32, device
+ *   stats   [n_layers, LASER_STATS_WORDS] int64 out, device; ACCUMULATED into when
+ *           accumulate != 0 (several batches), else overwritten:
+ *             0        tokens
+ *             1        sum of M_k          in units of 2^-32 (exact)
+ *             2        sum of the entropy  in units of 2^-32 (nats; each token rounded)
+ *             3, 4, 5  tokens in the regimes single-head, plateau, smooth
+ *             6        sum of n_near
+ *             7        sum of the best score s_max, in units of 2^-32 (exact)
+ *             8..71    histogram of M_k over 64 equal bins of [0, 1]; a dominance cutoff
+ *                      that sends a wanted share of tokens to the top-k branch is a
+ *                      quantile of it
+ *   means   [n_layers, 4] fp32 out, or NULL: mean M_k, mean entropy, mean s_max, mean n_near
+ *           of everything accumulated so far
+ * Scores are the routing softmax bit for bit; M_k is formed as in the routing rule (k best by
+ * logit descending, index ascending; fp32, left to right).  The paper names the regimes and
+ * gives no criterion; the one used counts the experts comparable to the best,
+ * n_near = #{i : s_i >= near_ratio * s_max} (the candidate-pool size for t_fix = near_ratio):
+ * single-head if n_near = 1, plateau if 2 <= n_near <= plateau_max, else smooth.
+ * Requires 1 <= k <= E <= LASER_MAX_EXPERTS, 0 <= near_ratio <= 1, plateau_max >= 1,
+ * 0 <= T, n_layers in 1..65535, T * n_layers tokens below 2^30; else LASER_ERR_INVALID_ARG.
+ * Enqueues a memset (unless accumulating) and up to two kernels on cuda_stream.
+ */
+#define LASER_STATS_WORDS 72
+int laser_score_stats(int32_t n_layers, int32_t T, int32_t E, int32_t k, const float* logits,
+                      float near_ratio, int32_t plateau_max, int32_t accumulate,
+                      int64_t* stats, float* means, void* cuda_stream);
+
 /* Size of the scratch array built into the library for laser_route_static (4 MiB). */
 enum { LASER_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 };
 

@@ -15,6 +15,11 @@
  *     (compile with -ffp-contract=off, no fast-math),
  *   - fmaf() is the correctly rounded fused multiply-add.
  *
+ * Parity unpinned by anything the paper prints (pinned by argument and by constructed
+ * cases only): the combine weights (the paper never mentions them), the granularity of
+ * the load update (no printed number depends on it), the RANDOM trimming convention
+ * (the paper names no generator or sampling procedure).
+ *
  * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
  */
 #include <math.h>

@@ -9,6 +9,7 @@
 #include "k12_fused.cuh"
 #include "k3_dispatch.cuh"
 #include "k4_metrics.cuh"
+#include "k5_score_stats.cuh"
 
 using namespace laser;
 
@@ -233,6 +234,45 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
 }  // namespace
 
 extern "C" int laser_version(void) { return 100; }
+
+static_assert(kStatsWords == LASER_STATS_WORDS, "header and kernel disagree");
+
+template <int N>
+static void launch_stats(dim3 grid, cudaStream_t st, int T, int E, int k, const float* logits,
+                         float near_ratio, int plateau_max, unsigned long long* stats) {
+  k5_score_stats<N><<<grid, kStatsThreads, 0, st>>>(T, E, k, logits, near_ratio, plateau_max,
+                                                    stats);
+}
+
+extern "C" int laser_score_stats(int32_t n_layers, int32_t T, int32_t E, int32_t k,
+                                 const float* logits, float near_ratio, int32_t plateau_max,
+                                 int32_t accumulate, int64_t* stats, float* means,
+                                 void* cuda_stream) {
+  if (n_layers < 1 || n_layers > 65535 || T < 0 || E < 1 || E > LASER_MAX_EXPERTS || k < 1 ||
+      k > E || !(near_ratio >= 0.0f && near_ratio <= 1.0f) || plateau_max < 1 || !stats ||
+      (T > 0 && !logits) || (long long)T * n_layers >= (1ll << 30))
+    return LASER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  auto* acc = reinterpret_cast<unsigned long long*>(stats);
+  if (!accumulate &&
+      cudaMemsetAsync(stats, 0, sizeof(int64_t) * kStatsWords * (size_t)n_layers, st) !=
+          cudaSuccess)
+    return LASER_ERR_CUDA;
+  if (T > 0) {
+    // blocks of 32 tokens per pass; about four waves of blocks over all layers
+    const int per_layer = (T + 31) / 32;
+    int gx = (4 * 148 * 8 + n_layers - 1) / n_layers;
+    if (per_layer <= 2 * gx) gx = per_layer;   // one pass each rather than an uneven second one
+    const dim3 grid(gx < 1 ? 1 : gx, n_layers);
+    if (E <= 8) launch_stats<8>(grid, st, T, E, k, logits, near_ratio, plateau_max, acc);
+    else if (E <= 32) launch_stats<32>(grid, st, T, E, k, logits, near_ratio, plateau_max, acc);
+    else if (E <= 64) launch_stats<64>(grid, st, T, E, k, logits, near_ratio, plateau_max, acc);
+    else if (E <= 128) launch_stats<128>(grid, st, T, E, k, logits, near_ratio, plateau_max, acc);
+    else launch_stats<256>(grid, st, T, E, k, logits, near_ratio, plateau_max, acc);
+  }
+  if (means) k5_stats_means<<<(n_layers + 127) / 128, 128, 0, st>>>(n_layers, acc, means);
+  return cudaGetLastError() == cudaSuccess ? LASER_OK : LASER_ERR_CUDA;
+}
 
 extern "C" int laser_imbalance(int32_t n_layers, int32_t E, int32_t n_bins, const int32_t* offsets,
                                const int32_t* expert_to_bin, const float* placement,

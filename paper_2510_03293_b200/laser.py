@@ -34,7 +34,8 @@ MAX_EXPERTS = 256
 
 EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_route",
            "laser_route_layers", "laser_route_layers_profiled", "laser_host_arena_bytes",
-           "laser_route_host", "laser_route_static", "laser_imbalance")
+           "laser_route_host", "laser_route_static", "laser_imbalance",
+           "laser_score_stats")
 
 
 class LaserParams(ctypes.Structure):
@@ -74,6 +75,12 @@ _lib.laser_route_static.restype = ctypes.c_int
 
 _lib.laser_imbalance.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.laser_imbalance.restype = ctypes.c_int
+
+
+_lib.laser_score_stats.argtypes = [_i32, _i32, _i32, _i32, _vp, ctypes.c_float, _i32, _i32, _vp,
+                                   _vp, _vp]
+_lib.laser_score_stats.restype = ctypes.c_int
+STATS_WORDS = 72
 
 
 class LaserError(RuntimeError):
@@ -236,6 +243,26 @@ def imbalance(offsets, n_bins: int, expert_to_bin=None, placement=None, stream=N
     if rc != OK:
         raise LaserError(rc)
     return I, Ib, agg
+
+
+def score_stats(logits, k: int, near_ratio: float = 0.5, plateau_max: int = 4, stats=None,
+                stream=None):
+    """laser_score_stats on logits [L, T, E] (torch CUDA fp32).  Pass the returned `stats`
+    [L, 72] int64 back in to accumulate further batches.  Returns (stats, means [L, 4])."""
+    import torch
+
+    L, T, E = logits.shape
+    dev = logits.device
+    accumulate = stats is not None
+    if stats is None:
+        stats = torch.empty((L, STATS_WORDS), dtype=torch.int64, device=dev)
+    means = torch.empty((L, 4), dtype=torch.float32, device=dev)
+    s = torch.cuda.current_stream(dev) if stream is None else stream
+    rc = _lib.laser_score_stats(L, T, E, k, _ptr(logits), near_ratio, plateau_max,
+                                int(accumulate), _ptr(stats), _ptr(means), s.cuda_stream)
+    if rc != OK:
+        raise LaserError(rc)
+    return stats, means
 
 
 def route_host(hidden, w_g, bias, loads, p: LaserParams, arena, *, expert_to_bin=None,

@@ -407,3 +407,42 @@ def test_imbalance_kernel_matches_the_fp64_figures(cuda_device):
         assert np.array_equal(I2.cpu().numpy(), I.cpu().numpy())
         assert np.allclose(Ib2.cpu().numpy(), ref2["I_bins"], rtol=2e-6, atol=0)
         assert abs(float(agg2[1]) - ref2["I_agg_bins"]) <= 4e-6 * ref2["I_agg_bins"]
+
+
+@pytest.mark.parametrize("T,E,k,near,pmax", [(1, 8, 2, 0.5, 3), (777, 8, 2, 0.5, 3),
+                                              (1000, 32, 4, 0.25, 6), (515, 64, 6, 0.3, 8),
+                                              (300, 13, 13, 1.0, 1), (260, 200, 8, 0.0, 200),
+                                              (129, 256, 8, 0.5, 16)])
+def test_score_statistics_match_the_oracle(cuda_device, T, E, k, near, pmax):
+    """Integer words (tokens, M_k and s_max sums, regimes, n_near, histogram) bit for bit; the
+    entropy sum within T units of 2^-32 for the per-token rounding plus 1e-9 relative for the
+    two double-precision logarithms."""
+    import torch
+
+    import oracle
+    from oracle import score_stats as st
+    from paper_2510_03293_b200 import laser
+
+    rng = np.random.default_rng(1000 * E + T)
+    Lr = 2
+    x = (rng.standard_normal((Lr, T, E)) * rng.choice([0.3, 2.0, 6.0], (Lr, T, 1))).astype(np.float32)
+    x[0, 0, :] = 0.0                       # a flat row
+    x[-1, -1, :] = 0.0; x[-1, -1, E // 2] = 50.0   # a one-hot row
+    xd = torch.from_numpy(x).to(cuda_device)
+    stats, means = laser.score_stats(xd, k, near, pmax)
+    stats2, means2 = laser.score_stats(xd, k, near, pmax, stats=stats.clone())
+    torch.cuda.synchronize()
+    got, got2 = stats.cpu().numpy(), stats2.cpu().numpy()
+    assert np.array_equal(got2, 2 * got)       # accumulation over two batches
+    for l in range(Lr):
+        ref = st.score_stats(x[l], oracle.softmax(x[l]), k, near, pmax)
+        g = got[l]
+        assert g[0] == T
+        assert g[1] == round(ref["mass_sum"] * 2**32) and g[7] == round(ref["smax_sum"] * 2**32)
+        assert abs(int(g[2]) - ref["entropy_sum"] * 2**32) <= T + 1e-9 * ref["entropy_sum"] * 2**32 + 1
+        assert g[3:6].tolist() == ref["regimes"] and g[6] == ref["near_sum"]
+        assert g[8:].tolist() == ref["mass_hist"]
+        m = means.cpu().numpy()[l]
+        want = [ref["mean_mass"], ref["mean_entropy"], ref["mean_smax"], ref["mean_near"]]
+        assert np.allclose(m, want, rtol=3e-7, atol=1e-9)
+    assert np.array_equal(means.cpu().numpy(), means2.cpu().numpy())

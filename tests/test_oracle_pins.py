@@ -442,3 +442,46 @@ def test_imbalance_stats_by_hand_and_limits():
     L = oracle.route(x, np.zeros(8, np.int32), 2, 8, 2.0, 0.0)[2]
     st = lit.imbalance_stats(L[None], np.arange(8) // 2, 4)
     assert st["I"][0] == 1.0 and st["MV"][0] == 0.0 and st["I_bins"][0] == 1.0
+
+
+# ---- score statistics ----------------------------------------------------------------------
+def test_score_stats_closed_forms_and_library_entropy():
+    import scipy.stats
+
+    from oracle import score_stats as st
+
+    # flat gate: M_k = k/E, entropy = ln E, every expert is near the top -> smooth
+    E, k = 8, 2
+    x = np.zeros((5, E), np.float32)
+    r = st.score_stats(x, oracle.softmax(x), k, 0.5, 3)
+    assert r["mean_mass"] == k / E and abs(r["mean_entropy"] - math.log(E)) < 1e-12
+    assert r["regimes"] == [0, 0, 5] and r["mean_near"] == E and r["mass_hist"][16] == 5
+    # one expert far ahead: M_k -> 1, entropy -> 0, single-head
+    x = np.zeros((3, E), np.float32); x[:, 5] = 60.0
+    r = st.score_stats(x, oracle.softmax(x), k, 0.5, 3)
+    assert r["mean_mass"] == 1.0 and r["mean_entropy"] < 1e-20 and r["regimes"] == [3, 0, 0]
+    assert r["mass_hist"][63] == 3 and r["mean_smax"] == 1.0
+    # a experts with logit ln(b) over a flat rest: closed forms for scores, M_k and entropy
+    a, b, E = 3, 16.0, 16
+    x = np.zeros((1, E), np.float32); x[0, [2, 7, 11]] = np.float32(math.log(b))
+    s = oracle.softmax(x)
+    Z = a * b + (E - a)
+    H = -(a * (b / Z) * math.log(b / Z) + (E - a) * (1 / Z) * math.log(1 / Z))
+    r = st.score_stats(x, s, 2, 0.5, 4)
+    assert abs(r["mean_mass"] - 2 * b / Z) < 1e-6 and abs(r["mean_entropy"] - H) < 1e-5
+    assert r["regimes"] == [0, 1, 0] and r["near_sum"] == a
+    # ... and with the plateau bound below a it counts as smooth
+    assert st.score_stats(x, s, 2, 0.5, 2)["regimes"] == [0, 0, 1]
+    # random rows: entropy against the library routine, M_k against a sort of the scores
+    x = _rand_logits(300, 32, 77, 2.0)
+    s = oracle.softmax(x)
+    r = st.score_stats(x, s, 4, 0.25, 6)
+    Href = sum(float(scipy.stats.entropy(s[t].astype(np.float64) / s[t].astype(np.float64).sum()))
+               for t in range(300))
+    assert abs(r["entropy_sum"] - Href) < 1e-3      # scores sum to 1 only within fp32 rounding
+    top4 = np.sort(s.astype(np.float64), axis=1)[:, -4:].sum()
+    assert abs(r["mass_sum"] - top4) < 300 * 4e-7
+    assert sum(r["regimes"]) == 300 and sum(r["mass_hist"]) == 300
+    # n_near is the candidate-pool size of the routing rule with t_fix = near_ratio
+    cs = oracle.route(x, np.zeros(32, np.int32), 1, 32, 2.0, 0.25)[3]
+    assert r["near_sum"] == int(np.asarray(cs).sum())
