@@ -19,14 +19,18 @@
 
 namespace laser {
 
-// Shared memory per warp: int32 base[E] | uint32 mask[E] | int32 pos[32*k] | uint8 pe[32*k]
+// Shared memory per warp: int32 base[E] | uint32 mask[E] | int32 pos[32*k] | int32 seen[32*k] |
+// uint8 pe[32*k]; per block, in front of the warps' parts: int32 lin[E] | int32 off[E+1]
 __host__ __device__ inline size_t k3_warp_smem_bytes(int E, int k) {
-  return align256(2 * sizeof(int32_t) * (size_t)E + sizeof(int32_t) * 32 * (size_t)k +
+  return align256(2 * sizeof(int32_t) * (size_t)E + 2 * sizeof(int32_t) * 32 * (size_t)k +
                   32 * (size_t)k);
+}
+__host__ __device__ inline size_t k3_block_smem_bytes(int E) {
+  return align256(sizeof(int32_t) * (2 * (size_t)E + 1));
 }
 __host__ __device__ inline int k3_warps_per_block(int E, int k) {
   const size_t per = k3_warp_smem_bytes(E, k);
-  int w = (int)((size_t)160 * 1024 / per);
+  int w = (int)(((size_t)160 * 1024 - k3_block_smem_bytes(E)) / per);
   return w > 8 ? 8 : (w < 1 ? 1 : w);
 }
 
@@ -36,14 +40,28 @@ __global__ void k3_dispatch(const RouteArgs A) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int warps = blockDim.x >> 5;
   const int g = blockIdx.x * warps + warp;
-  if (g >= A.lay.n_groups) return;
   const int k = A.k, c = A.c, E = A.E, T = A.T;
 
-  unsigned char* mine = k3_smem + (size_t)warp * k3_warp_smem_bytes(E, k);
+  // the layer's offsets and loads on entry (L_in = L_out - count), once per block
+  int32_t* lin_s = reinterpret_cast<int32_t*>(k3_smem);
+  int32_t* off_s = lin_s + E;
+  {
+    const int32_t* off_g = A.offsets + (size_t)layer * (E + 1);
+    const int32_t* Lout = A.loads + (size_t)layer * E;
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) {
+      off_s[e] = off_g[e];
+      if (e < E) lin_s[e] = Lout[e] - (off_g[e + 1] - off_g[e]);
+    }
+  }
+  __syncthreads();
+  if (g >= A.lay.n_groups) return;
+
+  unsigned char* mine = k3_smem + k3_block_smem_bytes(E) + (size_t)warp * k3_warp_smem_bytes(E, k);
   int32_t* base = reinterpret_cast<int32_t*>(mine);
   uint32_t* mask = reinterpret_cast<uint32_t*>(base + E);
   int32_t* pos = base + 2 * E;
-  uint8_t* pe = reinterpret_cast<uint8_t*>(pos + 32 * k);
+  int32_t* seen = pos + 32 * k;
+  uint8_t* pe = reinterpret_cast<uint8_t*>(seen + 32 * k);
 
   const unsigned char* ws = A.ws + (size_t)layer * A.ws_ls;
   const long long t = (long long)g * 32 + lane;
@@ -73,7 +91,7 @@ __global__ void k3_dispatch(const RouteArgs A) {
   if (!valid) return;
 
   const float* sc = reinterpret_cast<const float*>(ws + A.lay.cand_scores) + (size_t)t * c;
-  const int32_t* off = A.offsets + (size_t)layer * (E + 1);
+  const int32_t* off = off_s;
   int32_t* perm = A.perm + (size_t)layer * T * k;
   int32_t* ids = A.expert_ids + ((size_t)layer * T + t) * k;
   float* w = A.weights + ((size_t)layer * T + t) * k;
@@ -98,20 +116,21 @@ __global__ void k3_dispatch(const RouteArgs A) {
   } else {
     // load seen by rank j: L_in[e] + position; L_in = L_out - count.  Smaller (load, j) first.
     // (Relaxed variant: the assignments made before the token's chunk take the position's place.)
-    const int32_t* Lout = A.loads + (size_t)layer * E;
     const int32_t* gb0 = nullptr;
     if (A.G != 1)
       gb0 = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) +
             (size_t)(A.G == 0 ? 0 : ((t / A.G) * A.G) / 32) * E;
+    int32_t* myseen = seen + lane * k;
     for (int j = 0; j < k; ++j) {
       const int ej = mype[j];
-      const long long Lj = (long long)Lout[ej] - (off[ej + 1] - off[ej]) +
-                           (gb0 ? gb0[ej] : mypos[j]);
+      myseen[j] = lin_s[ej] + (gb0 ? gb0[ej] : mypos[j]);   // below 2^31: loads are int32
+    }
+    for (int j = 0; j < k; ++j) {
+      const int ej = mype[j];
+      const int32_t Lj = myseen[j];
       int slot = 0;
       for (int i = 0; i < k; ++i) {
-        const int ei = mype[i];
-        const long long Li = (long long)Lout[ei] - (off[ei + 1] - off[ei]) +
-                             (gb0 ? gb0[ei] : mypos[i]);
+        const int32_t Li = myseen[i];
         slot += (Li < Lj || (Li == Lj && i < j)) ? 1 : 0;
       }
       ids[slot] = ej;
