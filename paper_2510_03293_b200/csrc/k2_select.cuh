@@ -18,9 +18,11 @@
 //             memory, and a candidate's prefix count comes back by shuffle.
 //   E  > 32   one 32-bit "who chose me" mask per (warp, expert) in shared memory, maintained
 //             with atomics by the tokens that change, and their exclusive prefix over warps.
-//             When a batch has few decision tokens, only the other tokens are counted in
-//             parallel and warp 0 takes the decision tokens one after the other
-//             (lane = candidate), which is then cheaper than block-wide sweeps.
+//             Under the rule's own order the fixed point is not iterated: the tokens without
+//             a decision are counted in parallel, the load every candidate of every decision
+//             token would see without the batch's decisions is worked out in parallel, and
+//             warp 0 takes the decision tokens one after the other (lane = candidate), adding
+//             the decisions made so far.  The sweeps serve the relaxed granularities.
 // The candidates' keys (load << 5 | score rank) are sorted by a compile-time bitonic network
 // over CMAX registers; the first k give the choice in the order the method lists it.
 // Per group of 32 tokens the block stores how many assignments of this call preceded the
@@ -37,8 +39,8 @@ constexpr int kK2Warps = kK2Threads / 32;
 constexpr int kK2Batch = kK2Threads;     // tokens per batch, thread = token
 constexpr int kK2FastMaxLoad = 1 << 25;  // 32-bit keys (load << 5 | rank) stay below 2^31
 constexpr int kK2MaxSweeps = kK2Batch + 2;
-constexpr int kK2ChainMax = 16;          // E > 32: batches with this many decision tokens or fewer
-                                         // take them one after the other
+constexpr int kK2ChainMax = kK2Batch;    // E > 32, the rule's own order: batches with this many
+                                         // decision tokens or fewer take them one after the other
 constexpr long long kK2WaitCycles = 4000000000LL;  // give up a wait after ~2 s
 
 __host__ __device__ inline bool k2_fast_shape(int k, int c) { return c <= 32 && k <= 32; }
@@ -49,15 +51,18 @@ __host__ __device__ inline size_t k2_batch_bytes(int c) {
 // Shared memory of the selection role:
 //   int32 L[E] | int32 Lin[E] | uint64 keys[c] | int32 wtot[8][max(E,32)] |
 //   uint32 mask[8][E] | int32 excl[8][E] (E > 32) | uint8 chosen[256][32] (E > 32) |
-//   2 batch buffers (c*, candidate ids)
+//   chain mode (E > 32): int32 dexcl[8][E] | int32 dcnt[E] | lists | uint32 dseen[256][CMAX] |
+//   uint8 dcand[256][CMAX] | 2 batch buffers (c*, candidate ids)
 __host__ __device__ inline size_t k2_smem_bytes(int E, int c, int k) {
   const size_t Ew = E > 32 ? E : 32;
   size_t b = 3 * align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c) +
              align256(sizeof(int32_t) * kK2Warps * Ew);
   if (!k2_fast_shape(k, c)) return b;
-  if (E > 32)
+  if (E > 32) {
+    const size_t cmax = c <= 4 ? 4 : (c <= 8 ? 8 : (c <= 16 ? 16 : 32));   // the sorting width
     b += 3 * align256(sizeof(int32_t) * kK2Warps * E) + align256(sizeof(int32_t) * E) +
-         (size_t)kK2Batch * 32 + 512;
+         (size_t)kK2Batch * 32 + 512 + (size_t)kK2Batch * cmax * 5;
+  }
   return b + 2 * k2_batch_bytes(c);
 }
 
@@ -127,10 +132,13 @@ struct K2Smem {
   uint32_t* mask;    // [8][E]  E > 32: bit i = token i of the warp chose this expert
   int32_t* excl;     // [8][E]  E > 32: exclusive prefix of the mask popcounts over warps
   uint8_t* chosen;   // [256][32] E > 32: current choice of every token, key order
-  int32_t* dexcl;    // [8][E]  E > 32, chain mode: decisions of earlier warps per expert
+  int32_t* dexcl;    // [8][E]  E > 32, chain mode: decisions of each warp's tokens per expert
   int32_t* dcnt;     // [E]     E > 32, chain mode: decisions so far in the batch per expert
   uint8_t* dlist;    // [256]   E > 32, chain mode: the batch's decision tokens in order
   int32_t* dwarp;    // [8]     E > 32, chain mode: decision tokens per warp
+  uint32_t* dseen;   // [256][CMAX] E > 32, chain mode: per decision token and candidate the load
+                     //         seen without the batch's decisions (all ones: no candidate)
+  uint8_t* dcand;    // [256][CMAX] E > 32, chain mode: the candidates' experts
 };
 
 // One batch of up to 256 tokens, thread = token, run by the whole block.
@@ -239,18 +247,24 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
   uint32_t* mk = sm.mask + warp * E;
   uint8_t* ch = sm.chosen + tid * 32;
 
-  // Few decision tokens: the other tokens' increments are still counted in parallel, but the
-  // decision tokens are then taken one after the other by warp 0, lane = candidate, which
-  // costs about 650 cycles each -- less than two block-wide sweeps up to kK2ChainMax tokens.
+  // The rule's own order (strict) with decision tokens in the batch: the other tokens' increments
+  // are counted in parallel, every decision token works out in parallel the load each of its
+  // candidates would see without the decisions of this batch, and warp 0 then takes the decision
+  // tokens one after the other, lane = candidate: add the decisions so far for the candidate's
+  // expert, rank the keys with shuffles, the k smallest are the choice.  One step costs a
+  // shared-memory round trip and CMAX shuffles whatever the batch looks like, where the
+  // block-wide fixed point needs a sweep per link of the longest dependency chain.
   if (strict && any_dec && n_dec <= kK2ChainMax) {
     if (valid && !dec)
       for (int j = 0; j < k; ++j) atomicOr(&mk[my[j]], 1u << lane);
     const unsigned dmask = __ballot_sync(0xffffffffu, dec);
     if (lane == 0) sm.dwarp[warp] = __popc(dmask);
     for (int e = tid; e < E; e += kK2Threads) sm.dcnt[e] = 0;
+    for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.dexcl[i] = 0;
     __syncthreads();   // masks of the fixed tokens and the warps' decision counts are complete
+    int at = 0;        // position of this decision token among the batch's decision tokens
     if (dec) {
-      int at = __popc(dmask & below);
+      at = __popc(dmask & below);
       for (int w = 0; w < warp; ++w) at += sm.dwarp[w];
       sm.dlist[at] = (uint8_t)tid;
     }
@@ -262,55 +276,82 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
         run += __popc(sm.mask[w * E + e]);
       }
       sm.wtot[e] = run;
-      sm.dexcl[e] = 0;   // no decision precedes warp 0
     }
-    __syncthreads();
-    if (warp == 0) {
-      int cur_w = 0;
-      // candidate `lane` of decision token i: expert and the load it sees without the
-      // decisions of this batch; fetched one token ahead of the ranking
-      auto fetch = [&](int i, int& t, int& e, uint32_t& seen) {
-        t = sm.dlist[i];
-        const int w = t >> 5, l = t & 31;
-        const bool has = lane < (int)cs_s[t];
-        e = has ? (int)ids_s[t * c + lane] : -1;
-        seen = has ? (uint32_t)(sm.L[e] + sm.excl[w * E + e] +
-                                __popc(sm.mask[w * E + e] & ((1u << l) - 1)))
-                   : 0u;
-      };
-      int t_n, e_n;
-      uint32_t seen_n;
-      fetch(0, t_n, e_n, seen_n);
-      for (int i = 0; i < n_dec; ++i) {
-        const int t = t_n, e = e_n;
-        const uint32_t seen = seen_n;
-        if (i + 1 < n_dec) fetch(i + 1, t_n, e_n, seen_n);
-        const int w = t >> 5;
-        while (cur_w < w) {   // decisions made so far precede every token of the next warps
-          ++cur_w;
-          for (int x = lane; x < E; x += 32) sm.dexcl[cur_w * E + x] = sm.dcnt[x];
-        }
-        __syncwarp();
-        const uint32_t key = e >= 0 ? (((seen + (uint32_t)sm.dcnt[e]) << 5) | (uint32_t)lane)
-                                    : 0xffffffffu;
-        int cnt = 0;
+    __syncthreads();   // excl is complete
+    // With a handful of decision tokens warp 0 lists their candidates itself and writes their
+    // results itself, which saves two block barriers; otherwise every decision token does.
+    const bool few = n_dec * CMAX <= 64;
+    if (!few) {
+      if (dec) {
 #pragma unroll
-        for (int j = 0; j < CMAX; ++j) cnt += __shfl_sync(0xffffffffu, key, j) < key ? 1 : 0;
-        if (e >= 0 && cnt < k) {
-          sm.dcnt[e] += 1;   // the candidates of one token are distinct experts
-          sel[t * k + cnt] = (uint8_t)lane;
+        for (int r = 0; r < CMAX; ++r) {
+          const bool has = r < cs;
+          const int e = has ? (int)my[r] : 0;
+          sm.dseen[at * CMAX + r] =
+              has ? (uint32_t)(sm.L[e] + sm.excl[warp * E + e] + __popc(mk[e] & below))
+                  : 0xffffffffu;
+          sm.dcand[at * CMAX + r] = (uint8_t)e;
+        }
+      }
+      __syncthreads();   // every decision token's candidates and base loads are listed
+    }
+    uint8_t* dch = sm.chosen;   // [n_dec][k] chosen ranks in the order the method lists them
+    if (warp == 0) {
+      if (few) {
+        for (int it = lane; it < n_dec * CMAX; it += 32) {
+          const int i = it / CMAX, r = it - i * CMAX;
+          const int t = sm.dlist[i], w = t >> 5;
+          const bool has = r < (int)cs_s[t];
+          const int e = has ? (int)ids_s[t * c + r] : 0;
+          sm.dseen[it] = has ? (uint32_t)(sm.L[e] + sm.excl[w * E + e] +
+                                          __popc(sm.mask[w * E + e] & ((1u << (t & 31)) - 1)))
+                             : 0xffffffffu;
+          sm.dcand[it] = (uint8_t)e;
         }
         __syncwarp();
       }
-      while (cur_w < kK2Warps - 1) {
-        ++cur_w;
-        for (int x = lane; x < E; x += 32) sm.dexcl[cur_w * E + x] = sm.dcnt[x];
+      const bool mine = lane < CMAX;
+      uint32_t s_n = mine ? sm.dseen[lane] : 0xffffffffu;
+      int e_n = mine ? (int)sm.dcand[lane] : 0;
+      for (int i = 0; i < n_dec; ++i) {
+        const uint32_t s_i = s_n;
+        const int e = e_n;
+        if (mine && i + 1 < n_dec) {
+          s_n = sm.dseen[(i + 1) * CMAX + lane];
+          e_n = (int)sm.dcand[(i + 1) * CMAX + lane];
+        }
+        const bool has = s_i != 0xffffffffu;
+        const uint32_t key = has ? (((s_i + (uint32_t)sm.dcnt[e]) << 5) | (uint32_t)lane)
+                                 : 0xffffffffu;
+        int cnt = 0;
+#pragma unroll
+        for (int j = 0; j < CMAX; ++j) cnt += __shfl_sync(0xffffffffu, key, j) < key ? 1 : 0;
+        if (has && cnt < k) {
+          sm.dcnt[e] += 1;   // the candidates of one token are distinct experts
+          dch[i * k + cnt] = (uint8_t)lane;
+        }
+        __syncwarp();
+      }
+    }
+    if (!few) __syncthreads();   // dcnt and the chosen ranks are final
+    // chosen ranks out; dexcl[w][e] counts the decisions of warp w's tokens for expert e
+    if (!few || warp == 0) {
+      const int first = few ? lane : tid, step = few ? 32 : kK2Threads;
+      for (int idx = first; idx < n_dec * k; idx += step) {
+        const int i = idx / k, j = idx - i * k;
+        const int t = sm.dlist[i], r = dch[idx];
+        sel[t * k + j] = (uint8_t)r;
+        atomicAdd(&sm.dexcl[(t >> 5) * E + sm.dcand[i * CMAX + r]], 1);
       }
     }
     __syncthreads();
     for (int i = tid; i < kK2Warps * E; i += kK2Threads) {
-      const int e = i % E;
-      if ((i / E) * 32 < n_here) g_base[i] = sm.L[e] - sm.Lin[e] + sm.excl[i] + sm.dexcl[i];
+      const int w = i / E, e = i - w * E;
+      if (w * 32 < n_here) {
+        int32_t before = sm.excl[i];   // fixed tokens, then decisions, of the warps before w
+        for (int w2 = 0; w2 < w; ++w2) before += sm.dexcl[w2 * E + e];
+        g_base[i] = sm.L[e] - sm.Lin[e] + before;
+      }
     }
     __syncthreads();   // every thread has read the masks, excl, dexcl and sm.L of this batch
     for (int e = tid; e < E; e += kK2Threads) sm.L[e] += sm.wtot[e] + sm.dcnt[e];
@@ -455,6 +496,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   sm.wtot = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * kK2Warps * Ew);
   sm.mask = nullptr; sm.excl = nullptr; sm.chosen = nullptr;
   sm.dexcl = nullptr; sm.dcnt = nullptr; sm.dlist = nullptr; sm.dwarp = nullptr;
+  sm.dseen = nullptr; sm.dcand = nullptr;
   if (E > 32 && k2_fast_shape(k, c)) {
     sm.mask = reinterpret_cast<uint32_t*>(p);  p += align256(sizeof(int32_t) * kK2Warps * E);
     sm.excl = reinterpret_cast<int32_t*>(p);   p += align256(sizeof(int32_t) * kK2Warps * E);
@@ -463,6 +505,8 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
     sm.dcnt = reinterpret_cast<int32_t*>(p);   p += align256(sizeof(int32_t) * E);
     sm.dlist = p;                               p += 256;
     sm.dwarp = reinterpret_cast<int32_t*>(p);  p += 256;
+    sm.dseen = reinterpret_cast<uint32_t*>(p); p += (size_t)kK2Batch * CMAX * sizeof(uint32_t);
+    sm.dcand = p;                               p += (size_t)kK2Batch * CMAX;
   }
   unsigned char* bufs = p;
   const size_t buf_bytes = k2_batch_bytes(c);
@@ -533,6 +577,21 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       for (int i = lane; i < (nt * c + 15) / 16; i += 32)
         cp_async16(dst_ids + 16 * i, src_ids + 16 * i);
     };
+    // The last warp looks ahead for the router's flags: those of batch b + 1 are loaded while
+    // batch b - 1 is processed and first used a whole batch later, so the latency of the loads
+    // is not on the path of any batch.  (A flag seen unset is simply looked at again by the
+    // blocking wait.)
+    auto load_flags = [&](int b1) -> int {
+      int f = 1;
+      if (ready && b1 < n_batches) {
+        const int t1 = b1 * kK2Batch, n1 = min(kK2Batch, T - t1);
+        const int rt = t1 / router_rows + lane;      // at most 16 flags per batch
+        if (rt <= (t1 + n1 - 1) / router_rows) f = ld_acquire(ready + rt);
+      }
+      return f;
+    };
+    const bool looker = warp == kK2Warps - 1;
+    int flag_next = looker ? load_flags(1) : 1;   // flags of batch b + 1
     bool staged = false;   // batch b is already on its way into its buffer
     for (int b = 0; b < n_batches; ++b) {
       const int t0 = b * kK2Batch, nt = min(kK2Batch, T - t0);
@@ -550,15 +609,8 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
         }
         stage(b);
       }
-      // The last warp looks whether the router has already published the next batch: its flag
-      // loads are issued here and first used after the barrier, so their latency is hidden.
-      const bool look = warp == kK2Warps - 1 && b + 1 < n_batches;
-      int flag_next = 1;
-      if (look && ready) {
-        const int t1 = t0 + kK2Batch, n1 = min(kK2Batch, T - t1);
-        const int rt = t1 / router_rows + lane;      // at most 16 flags per batch
-        if (rt <= (t1 + n1 - 1) / router_rows) flag_next = ld_acquire(ready + rt);
-      }
+      const bool look = looker && b + 1 < n_batches;
+      const int flag_after = looker ? load_flags(b + 2) : 1;   // used in the next iteration
       cp_async_wait_all();
       __syncthreads();   // batch b is in shared memory
       if (look) {
@@ -566,6 +618,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
         if (okn) stage_by_warp(b + 1);
         if (lane == 0) s_next[b & 1] = okn ? 1 : 0;
       }
+      flag_next = flag_after;
       const unsigned char* buf = bufs + (size_t)(b & 1) * buf_bytes;
       k2_batch<CMAX, SMALL>(sm, reinterpret_cast<const uint16_t*>(buf),
                                    buf + align256((size_t)kK2Batch * sizeof(uint16_t)), nt, E, k,
