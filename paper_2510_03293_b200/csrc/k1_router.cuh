@@ -252,8 +252,19 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
   constexpr uint32_t IDX = N - 1;
   constexpr int SH = N == 64 ? 6 : 7;
   static_assert(N == 64 || N == 128, "index bits");
-  float xmax = row[0];
-  for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, row[i]);
+  // The row has N >= E readable columns (those from E on are ignored), so that every group of
+  // CL columns is loaded and exponentiated without a branch and the calls interleave.
+  float xmax;
+  {
+    float m[4] = {row[0], row[0], row[0], row[0]};
+    int i = 0;
+    for (; i + 4 <= E; i += 4) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) m[q] = fmaxf(m[q], row[i + q]);
+    }
+    for (; i < E; ++i) m[0] = fmaxf(m[0], row[i]);
+    xmax = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+  }
 
   float a[8];
 #pragma unroll
@@ -265,17 +276,19 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
 #pragma unroll 1
   for (int g0 = 0; g0 < E; g0 += CL) {
     uint32_t B[CL];
+    float xv[CL], ev[CL];
+#pragma unroll
+    for (int i = 0; i < CL; ++i) xv[i] = row[g0 + i];   // g0 + i < N
+#pragma unroll
+    for (int i = 0; i < CL; ++i) ev[i] = exp32(__fsub_rn(xv[i], xmax));
 #pragma unroll
     for (int i = 0; i < CL; ++i) {
       const int e = g0 + i;
-      B[i] = 0;
-      if (e < E) {
-        const float x = row[e];
-        a[i & 7] = __fadd_rn(a[i & 7], exp32(__fsub_rn(x, xmax)));
-        const uint32_t u = __float_as_uint(x);
-        const uint32_t o = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
-        B[i] = (o & ~IDX) | (IDX - (uint32_t)e);
-      }
+      const bool in = e < E;
+      a[i & 7] = __fadd_rn(a[i & 7], in ? ev[i] : 0.0f);   // a >= +0: adding +0 changes nothing
+      const uint32_t u = __float_as_uint(xv[i]);
+      const uint32_t o = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+      B[i] = in ? ((o & ~IDX) | (IDX - (uint32_t)e)) : 0u;
     }
     sort_desc<CL>(B);
     if (g0 == 0) {
@@ -308,23 +321,60 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
   }
   float Mk = 0.0f, thr = 0.0f;
   int mprime = 0;
+  float sv[CL];   // scores of all CL listed ranks at once (those from c on are not used)
+#pragma unroll
+  for (int r = 0; r < CL; ++r)
+    sv[r] = __fdiv_rn(exp32(__fsub_rn(row[IDX - (R[r] & IDX)], xmax)), Z);
 #pragma unroll
   for (int r = 0; r < CL; ++r) {
     if (r < c) {
-      const int bi = (int)(IDX - (R[r] & IDX));
-      const float s = __fdiv_rn(exp32(__fsub_rn(row[bi], xmax)), Z);
+      const float s = sv[r];
       if (r == 0) { thr = __fmul_rn(t_fix, s); Mk = s; }
       else if (r < k) Mk = __fadd_rn(Mk, s);
       if (s >= thr) ++mprime;
-      cand_ids[r] = (uint8_t)bi;
-      cand_scores[r] = s;
-      if (r < k) { expert_ids[r] = bi; weights[r] = s; }
     }
   }
   const bool top_k_branch = (Mk >= eps_high);
   *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
-  if (top_k_branch && renorm) {
-    for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
+  float wv[CL];   // combine weights of the k best
+#pragma unroll
+  for (int r = 0; r < CL; ++r) wv[r] = (top_k_branch && renorm) ? __fdiv_rn(sv[r], Mk) : sv[r];
+  // Records out.  With c = 8 and an even k (the shapes this epilogue mostly sees) a token's
+  // record is written with 8- and 16-byte stores: the stores of a warp go to 32 different
+  // sectors each, so their number is what costs.
+  if constexpr (CL == 8) {
+    // (the scratch records are 8 and 32 bytes per token in a 256-byte aligned workspace; the
+    // caller's id and weight arrays only promise 4-byte alignment, hence the test)
+    if (c == 8 && (k & 1) == 0 &&
+        ((reinterpret_cast<uintptr_t>(expert_ids) | reinterpret_cast<uintptr_t>(weights)) & 7) == 0) {
+      uint32_t lo = 0, hi = 0;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        lo |= (IDX - (R[r] & IDX)) << (8 * r);
+        hi |= (IDX - (R[r + 4] & IDX)) << (8 * r);
+      }
+      *reinterpret_cast<uint2*>(cand_ids) = make_uint2(lo, hi);
+      *reinterpret_cast<float4*>(cand_scores) = make_float4(sv[0], sv[1], sv[2], sv[3]);
+      *reinterpret_cast<float4*>(cand_scores + 4) = make_float4(sv[4], sv[5], sv[6], sv[7]);
+#pragma unroll
+      for (int r = 0; r < CL; r += 2) {
+        if (r < k) {
+          *reinterpret_cast<int2*>(expert_ids + r) =
+              make_int2((int)(IDX - (R[r] & IDX)), (int)(IDX - (R[r + 1] & IDX)));
+          *reinterpret_cast<float2*>(weights + r) = make_float2(wv[r], wv[r + 1]);
+        }
+      }
+      return;
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < CL; ++r) {
+    if (r < c) {
+      const int bi = (int)(IDX - (R[r] & IDX));
+      cand_ids[r] = (uint8_t)bi;
+      cand_scores[r] = sv[r];
+      if (r < k) { expert_ids[r] = bi; weights[r] = wv[r]; }
+    }
   }
 }
 

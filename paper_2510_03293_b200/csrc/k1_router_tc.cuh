@@ -222,7 +222,10 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
   __syncwarp();
 
   // ---- epilogue, all 8 warps ------------------------------------------------------------
-  const bool acc_ok = tc_mbar_wait(acc_bar, 0u, abort);
+  // One lane polls for the accumulator; everybody else sleeps in the block barrier, so that the
+  // issue slots of the SM go to the blocks that are scoring or issuing copies.
+  bool acc_ok = true;
+  if (warp == 2 && lane == 0) acc_ok = tc_mbar_wait(acc_bar, 0u, abort);
   if (__syncthreads_or(acc_ok ? 0 : 1)) {
     if (tid == 0 && A.status) atomicOr(A.status, 2);
   } else {

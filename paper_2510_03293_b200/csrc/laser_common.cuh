@@ -78,7 +78,6 @@ __device__ __forceinline__ int pair_rank(const uint16_t* cstar, const uint8_t* s
 //   y < -80 -> 0;  n = rint(y*log2e);  r = y - n*ln2 (two fma steps);
 //   degree-7 Taylor polynomial in Horner form;  result = p * 2^n.
 __device__ __forceinline__ float exp32(float y) {
-  if (y < -80.0f) return 0.0f;
   float n = rintf(__fmul_rn(y, __uint_as_float(0x3FB8AA3Bu)));
   float r = __fmaf_rn(n, -__uint_as_float(0x3F317200u), y);
   r = __fmaf_rn(n, -__uint_as_float(0x35BFBE8Eu), r);
@@ -90,8 +89,9 @@ __device__ __forceinline__ float exp32(float y) {
   p = __fmaf_rn(p, r, 0.5f);
   p = __fmaf_rn(p, r, 1.0f);
   p = __fmaf_rn(p, r, 1.0f);
-  int ni = __float2int_rn(n);                       // in [-116, 0]
-  return __fmul_rn(p, __int_as_float((ni + 127) << 23));
+  int ni = __float2int_rn(n);                       // in [-116, 0] for y >= -80
+  const float v = __fmul_rn(p, __int_as_float((ni + 127) << 23));
+  return y < -80.0f ? 0.0f : v;                     // a select, so that calls interleave
 }
 
 }  // namespace laser
