@@ -58,8 +58,9 @@ def workload_config(w, n_layers, n_copies=1):
 
 def launches_per_step(w, L) -> int:
     """Kernels the library enqueues per step, per group of at most 64 layers: the fused
-    router + selection kernel and the dispatch kernel."""
-    return 2 * ((L + 63) // 64)
+    router + selection kernel and the dispatch kernel (calls of at most 256 tokens have their
+    dispatch done inside the first kernel)."""
+    return (1 if w.T <= 256 else 2) * ((L + 63) // 64)
 
 
 def kernel_sources_digest() -> str:
@@ -549,7 +550,7 @@ def run_decode(args, w):
                      "traffic": None, "bytes_per_launch": bytes_per_pass / S,
                      "note": "latency-bound: 0.26 MB per call"},
         "routing": {"status_word": status},
-        "gpu_launches": 2 * S * args.steps, "clocks": clocks,
+        "gpu_launches": launches_per_step(w, 1) * S * args.steps, "clocks": clocks,
         "e2e": {"value": w.T / e2e_sec, "unit": UNIT, "ms_per_step": e2e_sec * 1e3 * S,
                 "us_per_call": e2e_sec * 1e6, "h2d_bytes_per_step": h2d * S,
                 "d2h_bytes_per_step": d2h * S, "calls_timed": int(h_hidden.shape[0])},

@@ -31,6 +31,7 @@
 // device-bin sums.
 #pragma once
 #include "laser_common.cuh"
+#include "k3_dispatch.cuh"
 
 namespace laser {
 
@@ -64,6 +65,13 @@ __host__ __device__ inline size_t k2_smem_bytes(int E, int c, int k) {
          (size_t)kK2Batch * 32 + 512 + (size_t)kK2Batch * cmax * 5;
   }
   return b + 2 * k2_batch_bytes(c);
+}
+
+// Calls of at most this many 32-token groups have their dispatch done by the selection block
+// itself (one launch less); its scratch lies behind L, Lin and Lvis in the selection's memory.
+constexpr int kFusedDispatchGroups = 8;
+__host__ __device__ inline size_t k2_fused_dispatch_bytes(int E, int k) {
+  return 3 * align256(sizeof(int32_t) * E) + (size_t)kK2Warps * k3_warp_smem_bytes(E, k);
 }
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
@@ -650,9 +658,10 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   int32_t before = 0;
   for (int w = 0; w < warp; ++w) before += s_warp_tot[w];
   int32_t* offsets = A.offsets + (size_t)layer * (E + 1);
+  __shared__ int32_t s_off[kMaxExperts + 1];
   if (tid < E) {
-    offsets[tid] = before + incl - cnt;
-    if (tid == E - 1) offsets[E] = before + incl;
+    offsets[tid] = s_off[tid] = before + incl - cnt;
+    if (tid == E - 1) offsets[E] = s_off[E] = before + incl;
   }
   if (A.bin_loads) {
     const int B = A.n_bins;
@@ -666,6 +675,15 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       }
       bl[b] += s;
     }
+  }
+  if (A.fuse_dispatch) {
+    // few groups: the dispatch of this layer here, instead of one more launch.  The barrier makes
+    // the offsets and this block's chosen ranks and group base counts visible to all its warps;
+    // the routers' records were acquired with their flags.
+    __syncthreads();
+    unsigned char* scratch = k2_smem + 3 * align256(sizeof(int32_t) * E);
+    for (int g = warp; g < n_groups; g += kK2Warps)
+      k3_group(A, layer, g, sm.Lin, s_off, scratch + (size_t)warp * k3_warp_smem_bytes(E, k));
   }
 }
 

@@ -34,29 +34,13 @@ __host__ __device__ inline int k3_warps_per_block(int E, int k) {
   return w > 8 ? 8 : (w < 1 ? 1 : w);
 }
 
-__global__ void k3_dispatch(const RouteArgs A) {
-  extern __shared__ __align__(16) unsigned char k3_smem[];
-  const int layer = A.layer0 + blockIdx.y;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int warps = blockDim.x >> 5;
-  const int g = blockIdx.x * warps + warp;
+// Group g (32 tokens) of absolute layer `layer`, by one warp.  lin_s / off_s: the layer's loads
+// on entry and its offsets in shared memory; mine: k3_warp_smem_bytes() of scratch for the warp.
+__device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
+                                         const int32_t* lin_s, const int32_t* off_s,
+                                         unsigned char* mine) {
+  const int lane = threadIdx.x & 31;
   const int k = A.k, c = A.c, E = A.E, T = A.T;
-
-  // the layer's offsets and loads on entry (L_in = L_out - count), once per block
-  int32_t* lin_s = reinterpret_cast<int32_t*>(k3_smem);
-  int32_t* off_s = lin_s + E;
-  {
-    const int32_t* off_g = A.offsets + (size_t)layer * (E + 1);
-    const int32_t* Lout = A.loads + (size_t)layer * E;
-    for (int e = threadIdx.x; e <= E; e += blockDim.x) {
-      off_s[e] = off_g[e];
-      if (e < E) lin_s[e] = Lout[e] - (off_g[e + 1] - off_g[e]);
-    }
-  }
-  __syncthreads();
-  if (g >= A.lay.n_groups) return;
-
-  unsigned char* mine = k3_smem + k3_block_smem_bytes(E) + (size_t)warp * k3_warp_smem_bytes(E, k);
   int32_t* base = reinterpret_cast<int32_t*>(mine);
   uint32_t* mask = reinterpret_cast<uint32_t*>(base + E);
   int32_t* pos = base + 2 * E;
@@ -144,6 +128,31 @@ __global__ void k3_dispatch(const RouteArgs A) {
   }
   if (A.renorm)
     for (int j = 0; j < k; ++j) w[j] = __fdiv_rn(w[j], sum);
+}
+
+__global__ void k3_dispatch(const RouteArgs A) {
+  extern __shared__ __align__(16) unsigned char k3_smem[];
+  const int layer = A.layer0 + blockIdx.y;
+  const int warp = threadIdx.x >> 5;
+  const int warps = blockDim.x >> 5;
+  const int g = blockIdx.x * warps + warp;
+  const int E = A.E;
+
+  // the layer's offsets and loads on entry (L_in = L_out - count), once per block
+  int32_t* lin_s = reinterpret_cast<int32_t*>(k3_smem);
+  int32_t* off_s = lin_s + E;
+  {
+    const int32_t* off_g = A.offsets + (size_t)layer * (E + 1);
+    const int32_t* Lout = A.loads + (size_t)layer * E;
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) {
+      off_s[e] = off_g[e];
+      if (e < E) lin_s[e] = Lout[e] - (off_g[e + 1] - off_g[e]);
+    }
+  }
+  __syncthreads();
+  if (g >= A.lay.n_groups) return;
+  k3_group(A, layer, g, lin_s, off_s,
+           k3_smem + k3_block_smem_bytes(E) + (size_t)warp * k3_warp_smem_bytes(E, A.k));
 }
 
 }  // namespace laser

@@ -34,10 +34,17 @@ int validate_params(const laser_params* p) {
   return LASER_OK;
 }
 
+// shared memory the selection role needs in a launch
+size_t selection_smem(const RouteArgs& a) {
+  const size_t b = k2_smem_bytes(a.E, a.c, a.k);
+  const size_t f = a.fuse_dispatch ? k2_fused_dispatch_bytes(a.E, a.k) : 0;
+  return b > f ? b : f;
+}
+
 template <int NT, int MT, int KU, int CMAX>
 cudaError_t launch_k12(const RouteArgs& a, int n_layers, cudaStream_t s) {
   size_t smem = router_smem_bytes(NT, MT);
-  const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
+  const size_t smem2 = selection_smem(a);
   if (smem2 > smem) smem = smem2;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k12_route_select<NT, MT, KU, CMAX>,
@@ -98,7 +105,7 @@ template <int N, int CMAX>
 cudaError_t launch_k12_tc(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
                           const CUtensorMap& mw, cudaStream_t s) {
   size_t smem = tc_smem_bytes<N>();
-  const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
+  const size_t smem2 = selection_smem(a);
   if (smem2 > smem) smem = smem2;
   cudaError_t e = cudaFuncSetAttribute(k12_route_select_tc<N, CMAX>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -142,7 +149,7 @@ bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, 
 template <int NT, int KU, int CMAX>
 cudaError_t launch_k12_splitk(const RouteArgs& a, int n_layers, cudaStream_t s) {
   size_t smem = router_splitk_smem_bytes(NT);
-  const size_t smem2 = k2_smem_bytes(a.E, a.c, a.k);
+  const size_t smem2 = selection_smem(a);
   if (smem2 > smem) smem = smem2;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k12_route_select_splitk<NT, KU, CMAX>,
@@ -224,6 +231,7 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   if (launch_k12_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
   if (!mark(1)) return LASER_ERR_CUDA;
   if (!mark(2)) return LASER_ERR_CUDA;
+  if (a.fuse_dispatch) return mark(3) ? LASER_OK : LASER_ERR_CUDA;   // done by the selection blocks
   const int warps = k3_warps_per_block(a.E, a.k);
   const size_t smem3 = k3_block_smem_bytes(a.E) + (size_t)warps * k3_warp_smem_bytes(a.E, a.k);
   if (smem3 > 48 * 1024 &&
@@ -360,6 +368,7 @@ extern "C" int laser_route_layers_profiled(
   a.T = p->T; a.d = p->d; a.E = p->E; a.k = p->k; a.c = p->c;
   a.n_bins = p->n_bins; a.renorm = p->renormalize ? 1 : 0;
   a.G = p->update_granularity;
+  a.fuse_dispatch = a.lay.n_groups <= kFusedDispatchGroups ? 1 : 0;
   a.trim_random = p->trim_mode == 1 ? 1 : 0;
   a.seed = p->seed;
   a.ld_h = p->ld_hidden; a.ld_w = p->ld_w;

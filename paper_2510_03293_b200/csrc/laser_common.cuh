@@ -61,6 +61,8 @@ struct RouteArgs {
                            // 0 or a multiple of 32 = relaxed variant (loads seen refreshed
                            // every G tokens, 0 = once per call)
   long long ld_h, ld_w;
+  int fuse_dispatch;       // 1 = the selection block also runs the dispatch of its layer (calls
+                           //     of a few groups), and no dispatch kernel is launched
   int layer0;              // first layer of this launch
   float eps_high[kMaxLayersPerLaunch];
   float t_fix[kMaxLayersPerLaunch];
