@@ -19,21 +19,25 @@ def to_dev_bf16(bits, dev):
 class Padded:
     """A device tensor with PAD sentinel elements on both sides of the payload."""
 
-    def __init__(self, shape, dtype, dev, fill):
+    def __init__(self, shape, dtype, dev, fill, skew=0):
         import torch
 
         n = int(np.prod(shape)) if len(shape) else 1
         self.fill = fill
-        self.buf = torch.full((n + 2 * PAD,), fill, dtype=dtype, device=dev)
-        self.view = self.buf[PAD:PAD + n].view(*shape)
+        self.buf = torch.full((n + 2 * PAD + skew,), fill, dtype=dtype, device=dev)
+        # skew = 1 puts a 4-byte type on an address that is not a multiple of 8
+        self.view = self.buf[PAD + skew:PAD + skew + n].view(*shape)
 
     def intact(self):
         b = self.buf
-        return bool((b[:PAD] == self.fill).all().item() and (b[-PAD:] == self.fill).all().item())
+        lo = self.view.data_ptr() - b.data_ptr()
+        lo //= b.element_size()
+        return bool((b[:lo] == self.fill).all().item() and
+                    (b[lo + self.view.numel():] == self.fill).all().item())
 
 
 def run_gpu(dev, hb, wb, bias, loads0, k, c, eps, tfix, renorm=1, n_bins=1, e2b=None,
-            bins0=None, want_logits=True):
+            bins0=None, want_logits=True, skew=0):
     """One laser_route call; returns dict of numpy outputs.  Checks the canaries."""
     import torch
 
@@ -47,8 +51,8 @@ def run_gpu(dev, hb, wb, bias, loads0, k, c, eps, tfix, renorm=1, n_bins=1, e2b=
     loads = torch.from_numpy(np.asarray(loads0, np.int32).copy()).to(dev)
     bins = None if bins0 is None else torch.from_numpy(np.asarray(bins0, np.int32).copy()).to(dev)
     pads = dict(
-        ids=Padded((1, T, k), torch.int32, dev, CANARY_I),
-        w=Padded((1, T, k), torch.float32, dev, CANARY_F),
+        ids=Padded((1, T, k), torch.int32, dev, CANARY_I, skew),
+        w=Padded((1, T, k), torch.float32, dev, CANARY_F, skew),
         off=Padded((1, E + 1), torch.int32, dev, CANARY_I),
         perm=Padded((1, T * k), torch.int32, dev, CANARY_I),
         logits=Padded((1, T, E), torch.float32, dev, CANARY_F),

@@ -446,3 +446,17 @@ def test_score_statistics_match_the_oracle(cuda_device, T, E, k, near, pmax):
         want = [ref["mean_mass"], ref["mean_entropy"], ref["mean_smax"], ref["mean_near"]]
         assert np.allclose(m, want, rtol=3e-7, atol=1e-9)
     assert np.array_equal(means.cpu().numpy(), means2.cpu().numpy())
+
+
+@pytest.mark.parametrize("router", ["tile", "splitk"])
+def test_id_and_weight_arrays_on_4_byte_boundaries(cuda_device, monkeypatch, router):
+    """The caller's id and weight arrays only have to be 4-byte aligned: the tensor-memory
+    router's 8-byte record stores must not be used then, and the results must not change."""
+    monkeypatch.setenv("LASER_ROUTER", router)
+    hb, wb, bias = layer(700, 512, 64, seed=31)
+    z = np.zeros(64, np.int32)
+    a = run_gpu(cuda_device, hb, wb, bias, z, 6, 8, 0.4, 0.8)
+    b = run_gpu(cuda_device, hb, wb, bias, z, 6, 8, 0.4, 0.8, skew=1)
+    for name in ("expert_ids", "weights", "offsets", "perm", "loads"):
+        assert np.array_equal(a[name], b[name]), name
+    check_against_oracle(b, hb, wb, bias, z, 6, 8, 0.4, 0.8)
