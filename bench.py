@@ -237,8 +237,10 @@ def run_gpu(args, w):
                           update_granularity=args.granularity,
                           trim_mode=0 if args.random_trim is None else 1,
                           seed=args.random_trim or 0)
-    loads = torch.zeros((L, w.E), dtype=torch.int32, device=dev)
-    bins = torch.zeros((L, w.n_bins), dtype=torch.int32, device=dev)
+    # load counters of experts and bins in one buffer, so that a step resets them with one memset
+    state = torch.zeros((L * (w.E + w.n_bins),), dtype=torch.int32, device=dev)
+    loads = state[:L * w.E].view(L, w.E)
+    bins = state[L * w.E:].view(L, w.n_bins)
     ws = torch.empty((laser.workspace_bytes(p) * L,), dtype=torch.uint8, device=dev)
     out = None
     exact_ids = exact_imb = None
@@ -263,7 +265,7 @@ def run_gpu(args, w):
 
     def step(events=None):
         nonlocal out, it
-        loads.zero_(); bins.zero_()
+        state.zero_()
         out = laser.route_layers(hiddens[it % n_copies], data["w_g"], data["bias"], loads, p,
                                  bin_loads=bins, eps_high=data["eps_high"], t_fix=data["t_fix"],
                                  out=out, workspace=ws, stage_events=events)
