@@ -34,11 +34,119 @@ __host__ __device__ inline int k3_warps_per_block(int E, int k) {
   return w > 8 ? 8 : (w < 1 ? 1 : w);
 }
 
+// k3_group for k <= KR with a token's experts, positions and seen loads in registers (every loop
+// over the k slots fully unrolled and guarded) instead of shared-memory arrays.
+template <int KR>
+__device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int g,
+                                              const int32_t* lin_s, const int32_t* off_s,
+                                              unsigned char* mine) {
+  const int lane = threadIdx.x & 31;
+  const int k = A.k, c = A.c, E = A.E, T = A.T;
+  int32_t* base = reinterpret_cast<int32_t*>(mine);
+  uint32_t* mask = reinterpret_cast<uint32_t*>(base + E);
+
+  const unsigned char* ws = A.ws + (size_t)layer * A.ws_ls;
+  const long long t = (long long)g * 32 + lane;
+  const bool valid = t < T;
+  const int cs = valid ? reinterpret_cast<const uint16_t*>(ws + A.lay.cstar)[t] : 0;
+  const uint8_t* cand = ws + A.lay.cand_ids + (size_t)t * c;
+  const uint8_t* sel = ws + A.lay.sel_rank + (size_t)t * k;
+  const int32_t* gb = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) + (size_t)g * E;
+
+  for (int e = lane; e < E; e += 32) { base[e] = gb[e]; mask[e] = 0; }
+  __syncwarp();
+  int ex[KR], rk[KR];   // expert and candidate rank of slot j as the selection listed them
+#pragma unroll
+  for (int j = 0; j < KR; ++j) { ex[j] = 0; rk[j] = j; }
+  if (valid) {
+#pragma unroll
+    for (int j = 0; j < KR; ++j)
+      if (j < k) {
+        if (cs > k) rk[j] = sel[j];
+        ex[j] = cand[rk[j]];
+        atomicOr(&mask[ex[j]], 1u << lane);
+      }
+  }
+  __syncwarp();
+  if (!valid) return;
+  const unsigned below = (1u << lane) - 1;
+  int pos[KR];
+#pragma unroll
+  for (int j = 0; j < KR; ++j) pos[j] = j < k ? base[ex[j]] + __popc(mask[ex[j]] & below) : 0;
+
+  const float* sc = reinterpret_cast<const float*>(ws + A.lay.cand_scores) + (size_t)t * c;
+  int32_t* perm = A.perm + (size_t)layer * T * k;
+  int32_t* ids = A.expert_ids + ((size_t)layer * T + t) * k;
+  float* w = A.weights + ((size_t)layer * T + t) * k;
+  const int32_t pair0 = (int32_t)(t * k);
+
+  if (cs == 0) {   // top-k branch: ids and weights were written by the router
+#pragma unroll
+    for (int j = 0; j < KR; ++j)
+      if (j < k) perm[off_s[ex[j]] + pos[j]] = pair0 + j;
+    return;
+  }
+  float v[KR];     // weights in slot order
+  int slot[KR];
+#pragma unroll
+  for (int j = 0; j < KR; ++j) { v[j] = 0.0f; slot[j] = j; }
+  if (cs > k) {
+#pragma unroll
+    for (int j = 0; j < KR; ++j)
+      if (j < k) v[j] = sc[rk[j]];
+  } else {
+    // c* == k: slots by (load seen, score rank); the load seen by rank j is L_in[e] + position
+    // (relaxed variant: + the assignments made before the token's chunk instead)
+    const int32_t* gb0 = nullptr;
+    if (A.G != 1)
+      gb0 = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) +
+            (size_t)(A.G == 0 ? 0 : ((t / A.G) * A.G) / 32) * E;
+    int32_t seen[KR];
+    float sj[KR];
+#pragma unroll
+    for (int j = 0; j < KR; ++j) {
+      seen[j] = j < k ? lin_s[ex[j]] + (gb0 ? gb0[ex[j]] : pos[j]) : 0;
+      sj[j] = j < k ? sc[j] : 0.0f;
+    }
+#pragma unroll
+    for (int j = 0; j < KR; ++j) {
+      int sl = 0;
+#pragma unroll
+      for (int i = 0; i < KR; ++i)
+        sl += (i < k && (seen[i] < seen[j] || (seen[i] == seen[j] && i < j))) ? 1 : 0;
+      slot[j] = sl;
+    }
+#pragma unroll
+    for (int s2 = 0; s2 < KR; ++s2) {
+#pragma unroll
+      for (int j = 0; j < KR; ++j)
+        if (j < k && slot[j] == s2) v[s2] = sj[j];
+    }
+  }
+  float sum = v[0];
+#pragma unroll
+  for (int j = 1; j < KR; ++j)
+    if (j < k) sum = __fadd_rn(sum, v[j]);
+#pragma unroll
+  for (int j = 0; j < KR; ++j)
+    if (j < k) {
+      ids[slot[j]] = ex[j];
+      perm[off_s[ex[j]] + pos[j]] = pair0 + slot[j];
+      w[j] = A.renorm ? __fdiv_rn(v[j], sum) : v[j];
+    }
+}
+
 // Group g (32 tokens) of absolute layer `layer`, by one warp.  lin_s / off_s: the layer's loads
 // on entry and its offsets in shared memory; mine: k3_warp_smem_bytes() of scratch for the warp.
 __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
                                          const int32_t* lin_s, const int32_t* off_s,
                                          unsigned char* mine) {
+  if (A.k <= 8) {   // unrolled to the smallest of 2, 4, 8 slots that holds k
+    if (A.k <= 2) k3_group_regs<2>(A, layer, g, lin_s, off_s, mine);
+    else if (A.k <= 4) k3_group_regs<4>(A, layer, g, lin_s, off_s, mine);
+    else k3_group_regs<8>(A, layer, g, lin_s, off_s, mine);
+    return;
+  }
   const int lane = threadIdx.x & 31;
   const int k = A.k, c = A.c, E = A.E, T = A.T;
   int32_t* base = reinterpret_cast<int32_t*>(mine);
