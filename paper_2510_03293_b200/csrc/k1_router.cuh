@@ -12,9 +12,11 @@
 
 namespace laser {
 
+// 16 bytes of hidden state, read once: not kept in L1, and fetched from memory 256 bytes at a
+// time (a hint: the rest of the 256 bytes is asked for by the neighbouring loads anyway).
 __device__ __forceinline__ uint4 ldg_stream(const uint16_t* p) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+  asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
