@@ -169,7 +169,8 @@ int laser_route_layers(int32_t n_layers,
  * stage_events is a HOST array of four cudaEvent_t handles (entries may be NULL),
  * recorded on cuda_stream: [0] before the first kernel, [1] and [2] after the kernel that
  * runs the contraction, the score epilogue and the ordered selection with its load update,
- * [3] after the dispatch kernels (which also write the combine weights).
+ * [3] after the dispatch kernels (which also write the combine weights).  Calls of at most 256
+ * tokens run their dispatch inside the first kernel: [3] then follows [2] directly.
  * With more than 64 layers the stages run once per group of 64 and the events keep the last
  * group's marks.  stage_events == NULL makes this identical to laser_route_layers.
  */
