@@ -89,3 +89,38 @@ def test_workspace_grows_with_the_trimming_size():
     large = laser.workspace_bytes(good(T=4096, c=8))
     assert large > small
     assert laser.host_arena_bytes(2, good()) > 2 * laser.workspace_bytes(good())
+
+
+def test_metric_entry_points_check_their_arguments_before_any_launch():
+    """laser_imbalance and laser_score_stats return INVALID_ARG for bad sizes and missing
+    pointers without touching the device (fake non-null pointers are never dereferenced)."""
+    import ctypes
+
+    lib = laser._lib
+    P = ctypes.c_void_p
+
+    def imb(L=2, E=8, B=4, off=4096, out=4096, placement=None):
+        return lib.laser_imbalance(L, E, B, P(off), None, P(placement) if placement else None,
+                                   P(out), None, None, None)
+
+    assert imb(L=0) == laser.ERR_INVALID_ARG
+    assert imb(L=70000) == laser.ERR_INVALID_ARG
+    assert imb(E=0) == laser.ERR_INVALID_ARG and imb(E=257) == laser.ERR_INVALID_ARG
+    assert imb(B=0) == laser.ERR_INVALID_ARG
+    assert imb(B=9) == laser.ERR_INVALID_ARG              # more bins than experts without a matrix
+    assert imb(B=2000, placement=4096) == laser.ERR_INVALID_ARG
+    assert imb(off=None) == laser.ERR_INVALID_ARG and imb(out=None) == laser.ERR_INVALID_ARG
+
+    def stats(L=2, T=64, E=8, k=2, x=4096, ratio=0.5, pmax=3, out=4096):
+        return lib.laser_score_stats(L, T, E, k, P(x), ctypes.c_float(ratio), pmax, 0, P(out),
+                                     None, None)
+
+    assert stats(L=0) == laser.ERR_INVALID_ARG
+    assert stats(T=-1) == laser.ERR_INVALID_ARG
+    assert stats(E=300) == laser.ERR_INVALID_ARG
+    assert stats(k=0) == laser.ERR_INVALID_ARG and stats(k=9) == laser.ERR_INVALID_ARG
+    assert stats(ratio=1.5) == laser.ERR_INVALID_ARG and stats(ratio=-0.1) == laser.ERR_INVALID_ARG
+    assert stats(ratio=float("nan")) == laser.ERR_INVALID_ARG
+    assert stats(pmax=0) == laser.ERR_INVALID_ARG
+    assert stats(x=None) == laser.ERR_INVALID_ARG and stats(out=None) == laser.ERR_INVALID_ARG
+    assert stats(L=65535, T=1 << 15) == laser.ERR_INVALID_ARG   # 2^30 tokens or more
