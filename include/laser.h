@@ -22,10 +22,7 @@
  *     before returning.
  *   - Return value: LASER_OK (0) or a negative status.  On a validation error nothing is
  *     launched and no output is touched.
- *   - The environment variable LASER_ROUTER (tile | splitk), read at every call, overrides the
- *     choice between the 128-token-tile routers and the 16-token split-K router, which is
- *     otherwise made from the number of tokens.  It changes speed, never results (logits may
- *     differ in the last bits, as between any two summation orders).  Meant for tests.
+ *   - The library reads no environment variable and keeps no routing state of its own.
  *   - Conditions only visible on the device are OR-ed into *status_word (device int32,
  *     may be NULL): LASER_DEV_LOAD_OVERFLOW, LASER_DEV_TIMEOUT.
  */
@@ -54,8 +51,10 @@ enum {
  * LOAD_OVERFLOW: on entry some load counter was negative or within T of 2^31-1, so it could
  *   overflow during the call.
  * TIMEOUT: the ordered selection runs in the same launch as the router and waits for the
- *   router's tiles; a wait gave up after about two seconds (it never should).
- * When either bit is set the call's results are unspecified. */
+ *   router's tiles; a wait gave up after about two seconds (it never should).  The layer is
+ *   then abandoned: its remaining selection and its dispatch are skipped, so that no stage reads
+ *   scratch records that were never written.
+ * When either bit is set the call's results are unspecified (every access stays in bounds). */
 enum { LASER_DEV_LOAD_OVERFLOW = 1, LASER_DEV_TIMEOUT = 2 };
 
 enum { LASER_MAX_EXPERTS = 256 };
@@ -122,7 +121,8 @@ int laser_workspace_bytes(const laser_params* p, size_t* bytes);
  *   w_g         [E, ld_w]      bf16, one row per expert, 16-byte aligned
  *   bias        [E] fp32 added to the logits, or NULL
  *   loads       [E] int32, in/out: L on entry, L + per-call counts on return
- *   expert_to_bin [E] int32 in [0, n_bins), or NULL for contiguous e / ceil(E / n_bins)
+ *   expert_to_bin [E] int32 in [0, n_bins), or NULL for contiguous e / ceil(E / n_bins);
+ *               an expert mapped outside that range is counted in no bin
  *   bin_loads   [n_bins] int32 in/out, or NULL to skip bin accounting
  *   p           host
  *   expert_ids  [T, k] int32 out.  Top-k branch: descending score.  Expanded branch:
@@ -167,10 +167,11 @@ int laser_route_layers(int32_t n_layers,
  * laser_route_layers that also records CUDA events between its stages, so that a caller can
  * time the router + selection kernel (stages 1-6) and the dispatch kernels (7) separately.
  * stage_events is a HOST array of four cudaEvent_t handles (entries may be NULL),
- * recorded on cuda_stream: [0] before the first kernel, [1] and [2] after the kernel that
- * runs the contraction, the score epilogue and the ordered selection with its load update,
- * [3] after the dispatch kernels (which also write the combine weights).  Calls of at most 256
- * tokens run their dispatch inside the first kernel: [3] then follows [2] directly.
+ * recorded on cuda_stream: [0] at the start, [1] after the scratch flags have been cleared and
+ * before the kernel that runs the contraction, the score epilogue and the ordered selection
+ * with its load update, [2] after that kernel, [3] after the dispatch kernel (which also
+ * writes the combine weights).  Small calls run their dispatch inside the first kernel: [3]
+ * then follows [2] directly.
  * With more than 64 layers the stages run once per group of 64 and the events keep the last
  * group's marks.  stage_events == NULL makes this identical to laser_route_layers.
  */
@@ -215,6 +216,7 @@ int laser_route_host(int32_t n_layers,
  *
  *   offsets       [n_layers, E+1] int32, as written by laser_route_layers
  *   expert_to_bin [E] int32 in [0, n_bins), or NULL for contiguous e / ceil(E / n_bins);
+ *                 an expert mapped outside that range is counted in no bin, as in laser_route;
  *                 ignored when placement is given
  *   placement     [n_bins, E] fp32 row-major, or NULL: the general matrix A (A[g,e] >= 0, each
  *                 column summing to 1; a replicated expert splits its tokens); not checked

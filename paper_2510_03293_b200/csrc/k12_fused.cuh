@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kK2Threads) k12_route_select(const RouteArgs A
       group_epilogue(A, local_layer, gtok0, tiles + (size_t)warp * 32 * LDS, LDS, lane);
   }
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0 && rt != A.withhold_tile) {
     int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
                                         A.lay.ready);
     __threadfence();
@@ -76,7 +76,7 @@ k12_route_select_splitk(const RouteArgs A, int n_layers) {
   const int rt = b / n_layers;
   router_splitk_block<NT, KU>(A, local_layer, rt, reinterpret_cast<float*>(dyn_smem));
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0 && rt != A.withhold_tile) {
     int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
                                         A.lay.ready);
     __threadfence();
@@ -104,13 +104,15 @@ k12_route_select_tc(const RouteArgs A, int n_layers, const __grid_constant__ CUt
   const int b = blockIdx.x - n_layers;
   const int local_layer = b % n_layers;
   const int rt = b / n_layers;
-  router_tc_block<N, (CMAX < 8 ? 8 : CMAX)>(A, &map_h, &map_w, local_layer, rt, dyn_smem);
-  // router_tc_block ends with a block barrier after the last record was written
-  if (threadIdx.x == 0) {
+  const bool done =
+      router_tc_block<N, (CMAX < 8 ? 8 : CMAX)>(A, &map_h, &map_w, local_layer, rt, dyn_smem);
+  // router_tc_block ends with a block barrier after the last record was written; a tile whose
+  // own waits ran out wrote no records and says so (-1), which aborts the layer's selection
+  if (threadIdx.x == 0 && rt != A.withhold_tile) {
     int* ready = reinterpret_cast<int*>(A.ws + (size_t)(A.layer0 + local_layer) * A.ws_ls +
                                         A.lay.ready);
     __threadfence();
-    st_release(ready + rt, 1);
+    st_release(ready + rt, done ? 1 : -1);
   }
 }
 

@@ -113,7 +113,7 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 //   the record lists the c* sampled experts in score-rank order.
 // Not a fast path: it ranks up to E experts round by round and keeps two byte arrays in local
 // memory.
-__device__ __noinline__ void token_epilogue_random(const float* row, int E, int k, int c,
+static __device__ __noinline__ void token_epilogue_random(const float* row, int E, int k, int c,
                                                    float eps_high, float t_fix, int renorm,
                                                    unsigned long long seed, int layer, long long t,
                                                    uint16_t* cstar, uint8_t* cand_ids,

@@ -135,8 +135,9 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
 
 // Router role of one block (256 threads) for tile `rt` (128 tokens) of local layer `layer`.
 // N: accumulator columns, a multiple of 16 with E <= N <= 256.
+// Returns false if one of the block's own waits ran out (no records were written then).
 template <int N, int CL>
-__device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtensorMap* map_h,
+__device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtensorMap* map_h,
                                                 const CUtensorMap* map_w, int layer, int rt,
                                                 unsigned char* dyn_smem) {
   constexpr int STAGES = tc_stages<N>();
@@ -164,8 +165,9 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   const int nk = (d + kTcSliceK - 1) / kTcSliceK;
-  const int row_h = abs_layer * T + rt * kTcTileM;   // rows of the [layers*T, d] view of hidden
-  const int row_w = abs_layer * E;                    // rows of the [layers*E, d] view of W_g
+  // rows of the [layers*T, d] and [layers*E, d] views (the launcher keeps both below 2^31)
+  const int row_h = abs_layer * T + rt * kTcTileM;
+  const int row_w = abs_layer * E;
   const int first_fill = nk < STAGES ? nk : STAGES;   // stage fills that need no free stage
 
   const bool has_bias = A.bias != nullptr;
@@ -236,7 +238,8 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
   // issue slots of the SM go to the blocks that are scoring or issuing copies.
   bool acc_ok = true;
   if (warp == 2 && lane == 0) acc_ok = tc_mbar_wait(acc_bar, 0u, abort);
-  if (__syncthreads_or(acc_ok ? 0 : 1)) {
+  const bool gave_up = __syncthreads_or(acc_ok ? 0 : 1) != 0;
+  if (gave_up) {
     if (tid == 0 && A.status) atomicOr(A.status, 2);
   } else {
     tc_fence_after();
@@ -369,6 +372,7 @@ __device__ __forceinline__ void router_tc_block(const RouteArgs& A, const CUtens
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                  ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
   }
+  return !gave_up;
 }
 
 }  // namespace laser

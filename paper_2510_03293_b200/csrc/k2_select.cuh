@@ -42,7 +42,7 @@ constexpr int kK2FastMaxLoad = 1 << 25;  // 32-bit keys (load << 5 | rank) stay 
 constexpr int kK2MaxSweeps = kK2Batch + 2;
 constexpr int kK2ChainMax = kK2Batch;    // E > 32, the rule's own order: batches with this many
                                          // decision tokens or fewer take them one after the other
-constexpr long long kK2WaitCycles = 4000000000LL;  // give up a wait after ~2 s
+constexpr long long kK2WaitCycles = 4000000000LL;  // default limit of a wait: ~2 s
 
 __host__ __device__ inline bool k2_fast_shape(int k, int c) { return c <= 32 && k <= 32; }
 __host__ __device__ inline size_t k2_batch_bytes(int c) {
@@ -91,18 +91,20 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 }
 // Called by one full warp: waits until the router blocks that produce tokens
 // [t_first, t_last] of this layer have published their records (the lanes share the flags).
-// Bounded: gives up after kK2WaitCycles and returns false.  block = false only tests once.
+// Bounded: gives up after `limit` cycles and returns false; also false as soon as one of the
+// tiles reports that it gave up itself (flag < 0).  block = false only tests once.
 __device__ __forceinline__ bool k2_wait_ready(const int* ready, int router_rows, int t_first,
-                                              int t_last, bool block = true) {
+                                              int t_last, long long limit, bool block = true) {
   const int lane = threadIdx.x & 31;
   const int rt0 = t_first / router_rows, rt1 = t_last / router_rows;
   const long long start = clock64();
   for (int base = rt0; base <= rt1; base += 32) {
     const int rt = base + lane;
     while (true) {
-      const bool set = rt > rt1 || ld_acquire(ready + rt) != 0;
-      if (__all_sync(0xffffffffu, set)) break;
-      if (!block || clock64() - start > kK2WaitCycles) return false;
+      const int v = rt > rt1 ? 1 : ld_acquire(ready + rt);
+      if (__any_sync(0xffffffffu, v < 0)) return false;
+      if (__all_sync(0xffffffffu, v != 0)) break;
+      if (!block || clock64() - start > limit) return false;
       __nanosleep(100);
     }
   }
@@ -490,6 +492,7 @@ template <int CMAX, bool SMALL>
 __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned char* k2_smem,
                                          const int* ready, int router_rows) {
   __shared__ int s_flag;      // outcome of a blocking wait for the router
+  __shared__ int s_gave_up;   // a wait ran out: the layer is aborted
   __shared__ int s_next[2];   // [b & 1]: batch b + 1 was prefetched during batch b
   const int E = A.E, k = A.k, c = A.c, T = A.T;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -529,6 +532,16 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
 
   if (sm.mask)
     for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
+  if (tid == 0) s_gave_up = 0;
+  // A wait that runs out (or a router tile that gave up) aborts the layer: the status bit is
+  // raised and the layer's abort word set, after which neither this block nor the dispatch
+  // reads the layer's scratch records again (they may be unwritten).
+  int* abort_word = const_cast<int*>(ready) + abort_word_index(T);
+  auto give_up = [&]() {
+    if (A.status) atomicOr(A.status, 2);
+    if (ready) st_release(abort_word, 1);
+    s_gave_up = 1;
+  };
   int too_big = 0;
   for (int e = tid; e < E; e += kK2Threads) {
     const int32_t v = g_loads[e];
@@ -546,8 +559,11 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       bool ok = true;
       for (int g = 0; g < n_groups && ok; ++g) {
         const int t0 = g * 32, n = min(32, T - t0);
-        if (ready && (t0 % router_rows) == 0) {
-          ok = k2_wait_ready(ready, router_rows, t0, min(T, t0 + router_rows) - 1);
+        // the whole group must be there: a router tile may be shorter than a group (16 tokens
+        // with the split-K router) or span several groups
+        if (ready && (router_rows < 32 || (t0 % router_rows) == 0)) {
+          ok = k2_wait_ready(ready, router_rows, t0, min(T, t0 + max(32, router_rows)) - 1,
+                             A.wait_cycles);
           if (!ok) break;
         }
         for (int e = lane; e < E; e += 32) g_base[(size_t)g * E + e] = sm.L[e] - sm.Lin[e];
@@ -558,7 +574,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
         k2_wide_group(sm.L, A.G == 1 ? sm.L : sm.Lvis, sm.keys, g_cs + t0, g_ids + (size_t)t0 * c,
                       g_sel + (size_t)t0 * k, n, k, c, lane);
       }
-      if (!ok && lane == 0 && A.status) atomicOr(A.status, 2);
+      if (!ok && lane == 0) give_up();
     }
   } else {
     const int n_batches = (T + kK2Batch - 1) / kK2Batch;
@@ -606,12 +622,12 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       if (!staged) {
         if (ready) {
           if (warp == 0) {
-            const bool good = k2_wait_ready(ready, router_rows, t0, t0 + nt - 1);
+            const bool good = k2_wait_ready(ready, router_rows, t0, t0 + nt - 1, A.wait_cycles);
             if (lane == 0) s_flag = good ? 1 : 0;
           }
           __syncthreads();
           if (!s_flag) {
-            if (tid == 0 && A.status) atomicOr(A.status, 2);
+            if (tid == 0) give_up();
             break;
           }
         }
@@ -622,7 +638,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       cp_async_wait_all();
       __syncthreads();   // batch b is in shared memory
       if (look) {
-        const bool okn = __all_sync(0xffffffffu, flag_next != 0);
+        const bool okn = __all_sync(0xffffffffu, flag_next > 0);
         if (okn) stage_by_warp(b + 1);
         if (lane == 0) s_next[b & 1] = okn ? 1 : 0;
       }
@@ -676,7 +692,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       bl[b] += s;
     }
   }
-  if (A.fuse_dispatch) {
+  if (A.fuse_dispatch && !s_gave_up) {   // (s_gave_up was written before the barriers above)
     // few groups: the dispatch of this layer here, instead of one more launch.  The barrier makes
     // the offsets and this block's chosen ranks and group base counts visible to all its warps;
     // the routers' records were acquired with their flags.

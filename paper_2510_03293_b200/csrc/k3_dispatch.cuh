@@ -238,6 +238,8 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
     for (int j = 0; j < k; ++j) w[j] = __fdiv_rn(w[j], sum);
 }
 
+// (defined in one translation unit only: the one that launches it)
+#ifdef LASER_DEFINE_K3_KERNEL
 __global__ void k3_dispatch(const RouteArgs A) {
   extern __shared__ __align__(16) unsigned char k3_smem[];
   const int layer = A.layer0 + blockIdx.y;
@@ -245,6 +247,10 @@ __global__ void k3_dispatch(const RouteArgs A) {
   const int warps = blockDim.x >> 5;
   const int g = blockIdx.x * warps + warp;
   const int E = A.E;
+  // a layer whose selection gave up a wait has unwritten scratch records: leave it alone
+  if (reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready)
+          [abort_word_index(A.T)] != 0)
+    return;
 
   // the layer's offsets and loads on entry (L_in = L_out - count), once per block
   int32_t* lin_s = reinterpret_cast<int32_t*>(k3_smem);
@@ -262,5 +268,6 @@ __global__ void k3_dispatch(const RouteArgs A) {
   k3_group(A, layer, g, lin_s, off_s,
            k3_smem + k3_block_smem_bytes(E) + (size_t)warp * k3_warp_smem_bytes(E, A.k));
 }
+#endif
 
 }  // namespace laser

@@ -76,8 +76,11 @@ k4_imbalance(int n_layers, int E, int n_bins, const int32_t* __restrict__ offset
         if (lane == 0) s_bin[g] = acc;
       }
     } else {
-      for (int e = threadIdx.x; e < E; e += kK4Threads)
-        atomicAdd(&s_ibin[e2b ? e2b[e] : e / per], s_cnt[e]);
+      for (int e = threadIdx.x; e < E; e += kK4Threads) {
+        // an expert mapped outside [0, n_bins) belongs to no bin, as in the routing kernel
+        const int b = e2b ? e2b[e] : e / per;
+        if (b >= 0 && b < n_bins) atomicAdd(&s_ibin[b], s_cnt[e]);
+      }
       __syncthreads();
       for (int b = threadIdx.x; b < n_bins; b += kK4Threads) s_bin[b] = (double)s_ibin[b];
     }

@@ -2,11 +2,10 @@
 // kernel selection by E, launches.  No allocation, no synchronisation (except the host-
 // buffer entry point), no state between calls.
 #include "../../include/laser.h"
+#include "../../include/laser_test_hooks.h"
 
-#include <cstdlib>
-#include <cstring>
-
-#include "k12_fused.cuh"
+#define LASER_DEFINE_K3_KERNEL
+#include "k12_launch.cuh"
 #include "k3_dispatch.cuh"
 #include "k4_metrics.cuh"
 #include "k5_score_stats.cuh"
@@ -14,6 +13,11 @@
 using namespace laser;
 
 namespace {
+
+// settings of include/laser_test_hooks.h (tests only; process-wide)
+int g_test_router = LASER_TEST_ROUTER_AUTO;
+int g_test_withhold_tile = -1;
+long long g_test_wait_cycles = 0;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -32,40 +36,6 @@ int validate_params(const laser_params* p) {
   if (p->ld_hidden % 8 != 0 || p->ld_w % 8 != 0) return LASER_ERR_MISALIGNED;
   if ((long long)p->T * p->k > 0x7fffffffLL) return LASER_ERR_INVALID_ARG;
   return LASER_OK;
-}
-
-// shared memory the selection role needs in a launch
-size_t selection_smem(const RouteArgs& a) {
-  const size_t b = k2_smem_bytes(a.E, a.c, a.k);
-  const size_t f = a.fuse_dispatch ? k2_fused_dispatch_bytes(a.E, a.k) : 0;
-  return b > f ? b : f;
-}
-
-template <int NT, int MT, int KU, int CMAX>
-cudaError_t launch_k12(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  size_t smem = router_smem_bytes(NT, MT);
-  const size_t smem2 = selection_smem(a);
-  if (smem2 > smem) smem = smem2;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k12_route_select<NT, MT, KU, CMAX>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
-  constexpr int RR = router_rows<NT, MT>();
-  const unsigned router_tiles = (unsigned)((a.T + RR - 1) / RR);
-  k12_route_select<NT, MT, KU, CMAX>
-      <<<n_layers * (1 + router_tiles), kK2Threads, smem, s>>>(a, n_layers);
-  return cudaGetLastError();
-}
-
-// The selection sorts CMAX >= c candidate keys in registers; pick the smallest network.
-template <int NT, int MT, int KU>
-cudaError_t launch_k12_for_c(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  constexpr int EP = NT * 8;
-  if (EP >= 4 && a.c <= 4) return launch_k12<NT, MT, KU, 4>(a, n_layers, s);
-  if (EP >= 8 && a.c <= 8) return launch_k12<NT, MT, KU, 8>(a, n_layers, s);
-  if (EP >= 16 && a.c <= 16) return launch_k12<NT, MT, KU, (EP >= 16 ? 16 : 8)>(a, n_layers, s);
-  return launch_k12<NT, MT, KU, (EP >= 32 ? 32 : EP)>(a, n_layers, s);
 }
 
 // ---- tensor-memory router (E > 32): TMA tensor maps and launch --------------------------
@@ -101,29 +71,6 @@ bool make_map(CUtensorMap* m, const void* base, long long rows, int d, long long
             promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int N, int CMAX>
-cudaError_t launch_k12_tc(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
-                          const CUtensorMap& mw, cudaStream_t s) {
-  size_t smem = tc_smem_bytes<N>();
-  const size_t smem2 = selection_smem(a);
-  if (smem2 > smem) smem = smem2;
-  cudaError_t e = cudaFuncSetAttribute(k12_route_select_tc<N, CMAX>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  const unsigned tiles = (unsigned)((a.T + kTcTileM - 1) / kTcTileM);
-  k12_route_select_tc<N, CMAX><<<n_layers * (1 + tiles), kK2Threads, smem, s>>>(a, n_layers, mh, mw);
-  return cudaGetLastError();
-}
-
-template <int N>
-cudaError_t launch_k12_tc_for_c(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
-                                const CUtensorMap& mw, cudaStream_t s) {
-  if (a.c <= 4) return launch_k12_tc<N, 4>(a, n_layers, mh, mw, s);
-  if (a.c <= 8) return launch_k12_tc<N, 8>(a, n_layers, mh, mw, s);
-  if (a.c <= 16) return launch_k12_tc<N, 16>(a, n_layers, mh, mw, s);
-  return launch_k12_tc<N, 32>(a, n_layers, mh, mw, s);
-}
-
 // Returns false if the tensor maps cannot be built for this call (the caller then uses the
 // warp-level router, which has no such requirement).
 bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, cudaError_t* err) {
@@ -132,6 +79,9 @@ bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, 
   const int N = a.E <= 64 ? 64 : (a.E <= 128 ? 128 : 256);
   CUtensorMap mh, mw;
   const long long total_layers = (long long)a.layer0 + n_layers;
+  // the kernels address rows of these views with signed 32-bit TMA coordinates
+  if (total_layers * a.T + kTcTileM > 0x7fffffffLL || total_layers * a.E > 0x7fffffffLL)
+    return false;
   // hidden states are fetched from memory 256 bytes at a time (two neighbouring 128-byte rows of
   // consecutive slices): measured 7.0 instead of 5.9 TB/s for this box shape on a plain stream
   if (!make_map(&mh, a.hidden, total_layers * a.T, a.d, a.ld_h, kTcTileM,
@@ -139,68 +89,40 @@ bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, 
     return false;
   if (!make_map(&mw, a.wg, total_layers * a.E, a.d, a.ld_w, N, CU_TENSOR_MAP_L2_PROMOTION_L2_128B))
     return false;
-  if (N == 64) *err = launch_k12_tc_for_c<64>(a, n_layers, mh, mw, s);
-  else if (N == 128) *err = launch_k12_tc_for_c<128>(a, n_layers, mh, mw, s);
-  else *err = launch_k12_tc_for_c<256>(a, n_layers, mh, mw, s);
+  if (N == 64) *err = launch_tc_n64(a, n_layers, mh, mw, s);
+  else if (N == 128) *err = launch_tc_n128(a, n_layers, mh, mw, s);
+  else *err = launch_tc_n256(a, n_layers, mh, mw, s);
   return true;
-}
-
-// ---- split-K router for calls with few tokens ---------------------------------------------
-template <int NT, int KU, int CMAX>
-cudaError_t launch_k12_splitk(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  size_t smem = router_splitk_smem_bytes(NT);
-  const size_t smem2 = selection_smem(a);
-  if (smem2 > smem) smem = smem2;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k12_route_select_splitk<NT, KU, CMAX>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
-  const unsigned tiles = (unsigned)((a.T + 15) / 16);
-  k12_route_select_splitk<NT, KU, CMAX>
-      <<<n_layers * (1 + tiles), kK2Threads, smem, s>>>(a, n_layers);
-  return cudaGetLastError();
-}
-
-template <int NT, int KU>
-cudaError_t launch_k12_splitk_for_c(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  constexpr int EP = NT * 8;
-  if (a.c <= 4) return launch_k12_splitk<NT, KU, 4>(a, n_layers, s);
-  if (a.c <= 8) return launch_k12_splitk<NT, KU, 8>(a, n_layers, s);
-  if (a.c <= 16) return launch_k12_splitk<NT, KU, (EP >= 16 ? 16 : 8)>(a, n_layers, s);
-  return launch_k12_splitk<NT, KU, (EP >= 32 ? 32 : EP)>(a, n_layers, s);
 }
 
 cudaError_t launch_k12_splitk_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
-  if (E <= 8) return launch_k12_splitk_for_c<1, 4>(a, n_layers, s);
-  if (E <= 16) return launch_k12_splitk_for_c<2, 4>(a, n_layers, s);
-  if (E <= 32) return launch_k12_splitk_for_c<4, 4>(a, n_layers, s);
-  if (E <= 64) return launch_k12_splitk_for_c<8, 2>(a, n_layers, s);
-  if (E <= 128) return launch_k12_splitk_for_c<16, 1>(a, n_layers, s);
-  return launch_k12_splitk_for_c<32, 1>(a, n_layers, s);
+  if (E <= 8) return launch_splitk_e8(a, n_layers, s);
+  if (E <= 16) return launch_splitk_e16(a, n_layers, s);
+  if (E <= 32) return launch_splitk_e32(a, n_layers, s);
+  if (E <= 64) return launch_splitk_e64(a, n_layers, s);
+  if (E <= 128) return launch_splitk_e128(a, n_layers, s);
+  return launch_splitk_e256(a, n_layers, s);
 }
 
 cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   const int E = a.E;
-  // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block.
-  // LASER_ROUTER=tile / splitk in the environment overrides the choice (testing aid).
+  // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block
+  // (laser_test_set_router overrides the choice for the tests)
   bool few = (long long)n_layers * ((a.T + 127) / 128) * 4 <= 148;
-  if (const char* f = std::getenv("LASER_ROUTER")) {
-    if (std::strcmp(f, "tile") == 0) few = false;
-    else if (std::strcmp(f, "splitk") == 0) few = true;
-  }
+  if (g_test_router == LASER_TEST_ROUTER_TILE) few = false;
+  else if (g_test_router == LASER_TEST_ROUTER_SPLITK) few = true;
   if (few) return launch_k12_splitk_for_E(a, n_layers, s);
   if (E > 32) {
     cudaError_t err = cudaSuccess;
     if (launch_k12_tensor_memory(a, n_layers, s, &err)) return err;
   }
-  if (E <= 8) return launch_k12_for_c<1, 1, 8>(a, n_layers, s);
-  if (E <= 16) return launch_k12_for_c<2, 2, 4>(a, n_layers, s);
-  if (E <= 32) return launch_k12_for_c<4, 2, 2>(a, n_layers, s);
-  if (E <= 64) return launch_k12_for_c<8, 2, 2>(a, n_layers, s);
-  if (E <= 128) return launch_k12_for_c<16, 1, 2>(a, n_layers, s);
-  return launch_k12_for_c<32, 1, 1>(a, n_layers, s);
+  if (E <= 8) return launch_warp_e8(a, n_layers, s);
+  if (E <= 16) return launch_warp_e16(a, n_layers, s);
+  if (E <= 32) return launch_warp_e32(a, n_layers, s);
+  if (E <= 64) return launch_warp_e64(a, n_layers, s);
+  if (E <= 128) return launch_warp_e128(a, n_layers, s);
+  return launch_warp_e256(a, n_layers, s);
 }
 
 // Enqueues all stages for layers [layer0, layer0 + n) of a batched call.
@@ -214,6 +136,8 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
     a.eps_high[l] = eps ? eps[layer0 + l] : p->eps_high;
     a.t_fix[l] = tfix ? tfix[layer0 + l] : p->t_fix;
   }
+  a.withhold_tile = g_test_withhold_tile;
+  a.wait_cycles = g_test_withhold_tile >= 0 ? g_test_wait_cycles : kK2WaitCycles;
   if (!mark(0)) return LASER_ERR_CUDA;
   if (a.T == 0) {
     // nothing to route: the call's offsets are all zero, loads and bins stay as they are
@@ -228,8 +152,8 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
                         (size_t)n, s) != cudaSuccess)
     return LASER_ERR_CUDA;
-  if (launch_k12_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
   if (!mark(1)) return LASER_ERR_CUDA;
+  if (launch_k12_for_E(a, n, s) != cudaSuccess) return LASER_ERR_CUDA;
   if (!mark(2)) return LASER_ERR_CUDA;
   if (a.fuse_dispatch) return mark(3) ? LASER_OK : LASER_ERR_CUDA;   // done by the selection blocks
   const int warps = k3_warps_per_block(a.E, a.k);
@@ -247,7 +171,23 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
 
 }  // namespace
 
-extern "C" int laser_version(void) { return 100; }
+extern "C" int laser_version(void) { return 200; }
+
+extern "C" int laser_test_set_router(int mode) {
+  if (mode != LASER_TEST_ROUTER_AUTO && mode != LASER_TEST_ROUTER_TILE &&
+      mode != LASER_TEST_ROUTER_SPLITK)
+    return -1;
+  const int prev = g_test_router;
+  g_test_router = mode;
+  return prev;
+}
+
+extern "C" int laser_test_withhold_tile(int tile, long long wait_cycles) {
+  if (tile >= 0 && wait_cycles < 1) return -1;
+  g_test_withhold_tile = tile < 0 ? -1 : tile;
+  g_test_wait_cycles = tile < 0 ? 0 : wait_cycles;
+  return 0;
+}
 
 static_assert(kStatsWords == LASER_STATS_WORDS, "header and kernel disagree");
 

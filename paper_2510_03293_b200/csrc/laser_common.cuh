@@ -17,6 +17,9 @@ struct WorkspaceLayout {
   size_t grp_base;     // int32  [n_groups, E]  per-expert count of this call's assignments made
                        //                   before the group (load at group start minus L_in)
   size_t ready;        // int32  [ceil(T/16)+1] router tiles published to the selection role
+                       //                   (1 = records written, -1 = the tile gave up); the last
+                       //                   word is the layer's abort word: non-zero once a wait ran
+                       //                   out, and then no later stage reads the layer's scratch
   size_t total;        // bytes per layer, multiple of 256
   int n_groups;        // ceil(T / 32): the ordered selection and the dispatch work on groups
                        // of 32 consecutive tokens
@@ -64,9 +67,14 @@ struct RouteArgs {
   int fuse_dispatch;       // 1 = the selection block also runs the dispatch of its layer (calls
                            //     of a few groups), and no dispatch kernel is launched
   int layer0;              // first layer of this launch
+  long long wait_cycles;   // limit of the selection's waits for the router, in clock cycles
+  int withhold_tile;       // test hook: the router tile with this index publishes no flag (-1: none)
   float eps_high[kMaxLayersPerLaunch];
   float t_fix[kMaxLayersPerLaunch];
 };
+
+// The layer's abort word (see WorkspaceLayout::ready).
+__host__ __device__ inline size_t abort_word_index(int T) { return (size_t)((T + 15) / 16); }
 
 // Rank position (in the score ranking) of slot j of token t as the selection left it:
 // tokens with c* > k were decided by the load-aware scan (sel_rank), all others keep their

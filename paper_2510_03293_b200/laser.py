@@ -30,12 +30,16 @@ ERR_CUDA = -5
 ERR_STATIC_SCRATCH = -6
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 DEV_LOAD_OVERFLOW = 1
+DEV_TIMEOUT = 2
 MAX_EXPERTS = 256
+ROUTER_AUTO, ROUTER_TILE, ROUTER_SPLITK = 0, 1, 2
 
 EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_route",
            "laser_route_layers", "laser_route_layers_profiled", "laser_host_arena_bytes",
            "laser_route_host", "laser_route_static", "laser_imbalance",
            "laser_score_stats")
+# include/laser_test_hooks.h: controls for the tests, not part of the routing interface
+TEST_EXPORTS = ("laser_test_set_router", "laser_test_withhold_tile")
 
 
 class LaserParams(ctypes.Structure):
@@ -81,12 +85,36 @@ _lib.laser_score_stats.argtypes = [_i32, _i32, _i32, _i32, _vp, ctypes.c_float, 
                                    _vp, _vp]
 _lib.laser_score_stats.restype = ctypes.c_int
 STATS_WORDS = 72
+_lib.laser_test_set_router.argtypes = [ctypes.c_int]
+_lib.laser_test_set_router.restype = ctypes.c_int
+_lib.laser_test_withhold_tile.argtypes = [ctypes.c_int, ctypes.c_longlong]
+_lib.laser_test_withhold_tile.restype = ctypes.c_int
 
 
 class LaserError(RuntimeError):
     def __init__(self, status: int):
         self.status = status
         super().__init__(f"laser: {strerror(status)} ({status})")
+
+
+def test_set_router(mode: int) -> int:
+    """laser_test_set_router: ROUTER_AUTO / ROUTER_TILE / ROUTER_SPLITK; returns the previous
+    mode.  For tests."""
+    prev = int(_lib.laser_test_set_router(int(mode)))
+    if prev < 0:
+        raise ValueError("unknown router mode %r" % (mode,))
+    return prev
+
+
+def test_withhold_tile(tile: int, wait_cycles: int = 0) -> None:
+    """laser_test_withhold_tile: router tile `tile` publishes no ready flag and the selection's
+    waits give up after `wait_cycles` clock cycles; tile < 0 restores.  For tests."""
+    if int(_lib.laser_test_withhold_tile(int(tile), int(wait_cycles))) != 0:
+        raise ValueError("wait_cycles must be positive")
+
+
+test_set_router.__test__ = False          # not pytest cases, whatever the names suggest
+test_withhold_tile.__test__ = False
 
 
 def version() -> int:

@@ -11,20 +11,40 @@ from paper_2510_03293_b200 import laser
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def declared_functions():
-    text = open(os.path.join(ROOT, "include", "laser.h")).read()
+def declared_functions(header="laser.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(laser_[a-z_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["laser.h", "laser_test_hooks.h"]
     names = declared_functions()
     assert set(names) == set(laser.EXPORTS)
+    hooks = declared_functions("laser_test_hooks.h")
+    assert set(hooks) == set(laser.TEST_EXPORTS)
     lib = ctypes.CDLL(laser.LIB_PATH)
-    for n in names:
+    for n in names + hooks:
         assert hasattr(lib, n), n
     assert laser.version() >= 100
     assert laser.strerror(0) == "ok" and "unknown" in laser.strerror(-99)
+
+
+def test_hooks_reject_bad_settings_and_restore():
+    assert laser.test_set_router(laser.ROUTER_TILE) == laser.ROUTER_AUTO
+    assert laser.test_set_router(laser.ROUTER_AUTO) == laser.ROUTER_TILE
+    with pytest.raises(ValueError):
+        laser.test_set_router(7)
+    assert laser.test_set_router(laser.ROUTER_AUTO) == laser.ROUTER_AUTO   # unchanged by the bad call
+    with pytest.raises(ValueError):
+        laser.test_withhold_tile(0, 0)
+    laser.test_withhold_tile(-1)
+
+
+def test_no_environment_lookups_in_the_library_sources():
+    csrc = os.path.join(ROOT, "paper_2510_03293_b200", "csrc")
+    for name in os.listdir(csrc):
+        assert "getenv" not in open(os.path.join(csrc, name)).read(), name
 
 
 def good(**over):

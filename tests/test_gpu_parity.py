@@ -10,6 +10,19 @@ from gpu_util import check_against_oracle, run_gpu, to_dev_bf16
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture
+def force_router():
+    """Selects the router by hand for one test (small shapes otherwise always take the
+    split-K router) and restores the automatic choice afterwards."""
+    from paper_2510_03293_b200 import laser
+
+    def choose(name):
+        laser.test_set_router({"tile": laser.ROUTER_TILE, "splitk": laser.ROUTER_SPLITK}[name])
+
+    yield choose
+    laser.test_set_router(laser.ROUTER_AUTO)
+
+
 def layer(T, d, E, seed, sigma=0.02, alpha=1.2, with_bias=True):
     return synth.make_layer(T, d, E, sigma, alpha, seed=seed, stream=E * 7 + d, with_bias=with_bias)
 
@@ -59,9 +72,9 @@ def test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B):
 
 
 @pytest.mark.parametrize("T,d,E,k,c,eps,tfix,renorm,B", [c_ for c_ in CASES if c_[0] < 4000])
-def test_small_cases_through_the_tile_routers(cuda_device, monkeypatch, T, d, E, k, c, eps, tfix,
+def test_small_cases_through_the_tile_routers(cuda_device, force_router, T, d, E, k, c, eps, tfix,
                                               renorm, B):
-    monkeypatch.setenv("LASER_ROUTER", "tile")
+    force_router("tile")
     test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B)
 
 
@@ -233,9 +246,9 @@ def _route_layers_strided(dev, hb, wb, bias, ld_h, ld_w, k, c, eps, tfix, B):
     (2, 150, 256, 256, 8, 16, 320, 256),    # ... 256 accumulator columns, two-pass epilogue
     (3, 300, 264, 8, 2, 4, 272, 280),       # warp-level router with padded rows
 ])
-def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, monkeypatch, router, L, T, d, E,
+def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, force_router, router, L, T, d, E,
                                                    k, c, ld_h, ld_w):
-    monkeypatch.setenv("LASER_ROUTER", router)   # both routers on the same small inputs
+    force_router(router)   # both routers on the same small inputs
     layers = [layer(T, d, E, seed=200 + l + E, sigma=0.05) for l in range(L)]
     hb = np.stack([x[0] for x in layers]); wb = np.stack([x[1] for x in layers])
     bias = np.stack([x[2] for x in layers])
@@ -306,9 +319,9 @@ def _run_relaxed(dev, hb, wb, bias, loads0, k, c, eps, tfix, G, B):
     (700, 128, 256, 8, 40, 0.30, 0.10),  # one-warp scan (candidate sets wider than a warp)
 ])
 @pytest.mark.parametrize("G", [0, 32, 96, 256, 1024])
-def test_relaxed_granularity_matches_its_oracle(cuda_device, monkeypatch, router, T, d, E, k, c,
+def test_relaxed_granularity_matches_its_oracle(cuda_device, force_router, router, T, d, E, k, c,
                                                 eps, tfix, G):
-    monkeypatch.setenv("LASER_ROUTER", router)
+    force_router(router)
     hb, wb, bias = layer(T, d, E, seed=400 + E + G, sigma=0.05)
     loads0 = np.random.default_rng(G + E).integers(0, 4, E).astype(np.int32)
     B = 4
@@ -335,13 +348,13 @@ def test_relaxed_granularity_matches_its_oracle(cuda_device, monkeypatch, router
     (600, 128, 100, 5, 12, 0.5, 0.2),    # 128 columns
     (500, 128, 256, 8, 16, 0.3, 0.3),    # 256 columns (two-pass epilogue)
 ])
-def test_random_trimming_matches_its_oracle(cuda_device, monkeypatch, router, T, d, E, k, c, eps,
+def test_random_trimming_matches_its_oracle(cuda_device, force_router, router, T, d, E, k, c, eps,
                                             tfix):
     import torch
 
     from paper_2510_03293_b200 import laser
 
-    monkeypatch.setenv("LASER_ROUTER", router)
+    force_router(router)
     dev = cuda_device
     Lr, B, seed = 2, 4, 0xC0FFEE1234
     layers = [layer(T, d, E, seed=500 + l + E, sigma=0.08) for l in range(Lr)]
@@ -449,10 +462,10 @@ def test_score_statistics_match_the_oracle(cuda_device, T, E, k, near, pmax):
 
 
 @pytest.mark.parametrize("router", ["tile", "splitk"])
-def test_id_and_weight_arrays_on_4_byte_boundaries(cuda_device, monkeypatch, router):
+def test_id_and_weight_arrays_on_4_byte_boundaries(cuda_device, force_router, router):
     """The caller's id and weight arrays only have to be 4-byte aligned: the tensor-memory
     router's 8-byte record stores must not be used then, and the results must not change."""
-    monkeypatch.setenv("LASER_ROUTER", router)
+    force_router(router)
     hb, wb, bias = layer(700, 512, 64, seed=31)
     z = np.zeros(64, np.int32)
     a = run_gpu(cuda_device, hb, wb, bias, z, 6, 8, 0.4, 0.8)

@@ -32,10 +32,14 @@ def route_static_once(dev, hb, wb, bias, loads0, bins0, k, c, eps, tfix, renorm,
         loads, bins,
         torch.full((T, E), -7.0, dtype=torch.float32, device=dev),
         torch.zeros((1,), dtype=torch.int32, device=dev))
-    laser.route_static(to_dev_bf16(hb, dev), to_dev_bf16(wb, dev), torch.from_numpy(bias).to(dev),
-                       loads, p, out, bin_loads=bins)
+    hidden, wg, bias_d = to_dev_bf16(hb, dev), to_dev_bf16(wb, dev), torch.from_numpy(bias).to(dev)
     torch.cuda.synchronize()
-    return dict(expert_ids=out.expert_ids.cpu().numpy(), weights=out.weights.cpu().numpy(),
+    free_before = torch.cuda.mem_get_info(dev)[0]      # the driver's own count of free bytes
+    laser.route_static(hidden, wg, bias_d, loads, p, out, bin_loads=bins)
+    torch.cuda.synchronize()
+    free_after = torch.cuda.mem_get_info(dev)[0]
+    return dict(free_before=free_before, free_after=free_after,
+                expert_ids=out.expert_ids.cpu().numpy(), weights=out.weights.cpu().numpy(),
                 offsets=out.offsets.cpu().numpy(), perm=out.perm.cpu().numpy(),
                 loads=loads.cpu().numpy(), bin_loads=bins.cpu().numpy(),
                 logits=out.logits.cpu().numpy(), status=int(out.status.item()))
@@ -62,6 +66,10 @@ def test_static_scratch_entry_matches_laser_route_twice_in_a_row(cuda_device):
         assert np.array_equal(got["weights"].view(np.uint32), want["weights"].view(np.uint32))
         assert np.array_equal(got["logits"].view(np.uint32), want["logits"].view(np.uint32))
         assert int(got["offsets"][-1]) == T * k
+        if i > 0:
+            # nothing was allocated or freed on the device by the call itself (the first call
+            # on a device may still load the kernels' code, so only later calls are held to it)
+            assert got["free_after"] == got["free_before"], (got["free_before"], got["free_after"])
 
 
 def test_static_scratch_entry_refuses_shapes_beyond_its_array(cuda_device):
