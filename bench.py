@@ -8,10 +8,14 @@ step.  Inputs are seeded synthetic tensors (4.3 GB of hidden states, larger than
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
-Prints one JSON line.  With --impl reference the CPU oracle is timed on the host cores on a
-bounded sample of the same workload.  --workload decode runs the decode stream (4096 successive
-64-token calls with the load state carried along) as one replayed CUDA graph and reports the
-latency per call.
+Prints one JSON line.  Without --workload the line is the Mixtral-shaped workload's, and its
+"workloads" key carries the same measurements for the other four shapes (tiny, DeepSeek-shaped,
+decode stream, E = 256 stress), each with its roofline fraction, routing statistics and the
+agreement with the CPU oracle run on its own logits.  With --impl reference the CPU oracle is
+timed on the host cores on a bounded sample of the same workload.  --workload decode runs the
+decode stream (4096 successive 64-token calls with the load state carried along) as one replayed
+CUDA graph and reports the latency per call.  --gpus N without a torchrun environment starts N
+replica processes itself.
 """
 from __future__ import annotations
 
@@ -54,6 +58,9 @@ def workload_config(w, n_layers, n_copies=1):
             (w.name, n_layers, w.T, w.d, w.E, w.k, w.c, w.n_bins),
             "tokens_per_step": n_layers * w.T, "t_fix": w.t_fix, "eps_high": list(w.eps_high),
             "cache": cache}
+
+
+DECODE_NODES_PER_CALL = 2   # a memset of the router's flags and one kernel
 
 
 def launches_per_step(w, L) -> int:
@@ -215,22 +222,61 @@ def aggregate_replicas(total_ms, steps, tokens_per_rank, dist, device):
     return ms_per_step, world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
-def run_gpu(args, w):
+class Context:
+    """Rank, device and (for N > 1 replicas) the process group of this process."""
+
+    def __init__(self):
+        import torch
+
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=self.dev)
+            self.dist = dist
+
+    def barrier(self):
+        import torch
+
+        if self.dist is not None:
+            self.dist.barrier()
+        torch.cuda.synchronize()
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.barrier()
+            self.dist.destroy_process_group()
+
+
+def new_events(torch, n):
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+    for e in evs:
+        e.record()
+    return evs
+
+
+def percentile(v, q):
+    s = sorted(v)
+    pos = (len(s) - 1) * q
+    lo = int(pos)
+    hi = min(lo + 1, len(s) - 1)
+    return s[lo] + (s[hi] - s[lo]) * (pos - lo)
+
+
+def run_layers(args, w, ctx, full):
+    """One workload of independent layers.  full: also the end-to-end leg, the CPU baseline
+    leg and the sustained loop (the headline workload); otherwise the device-timed figures,
+    the routing statistics and the oracle sample only."""
     import numpy as np
     import torch
 
     from paper_2510_03293_b200 import laser, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-
+    dev, dist, rank, world = ctx.dev, ctx.dist, ctx.rank, ctx.world
     L = w.layers if args.layers is None else args.layers
     data = synth.make_workload_torch(w, dev, seed=args.seed + rank, layers=L)
     p = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize, w.n_bins,
@@ -263,45 +309,40 @@ def run_gpu(args, w):
     hiddens = [data["hidden"]] + [data["hidden"].clone() for _ in range(n_copies - 1)]
     it = 0
 
-    def step(events=None):
+    def step(events=None, eps=None):
         nonlocal out, it
         state.zero_()
         out = laser.route_layers(hiddens[it % n_copies], data["w_g"], data["bias"], loads, p,
-                                 bin_loads=bins, eps_high=data["eps_high"], t_fix=data["t_fix"],
-                                 out=out, workspace=ws, stage_events=events)
+                                 bin_loads=bins, eps_high=data["eps_high"] if eps is None else eps,
+                                 t_fix=data["t_fix"], out=out, workspace=ws, stage_events=events)
         it += 1
 
-    def new_events(n):
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
-        for e in evs:
-            e.record()
-        return evs
+    def timed_steps(n, eps=None):
+        """n steps with their stage events; returns (total ms, per-step stage events)."""
+        stage = [new_events(torch, 4) for _ in range(n)]
+        t_begin, t_end = new_events(torch, 2)
+        ctx.barrier()
+        t_begin.record()
+        for i in range(n):
+            step(stage[i], eps)
+        t_end.record()
+        ctx.barrier()
+        return t_begin.elapsed_time(t_end), stage
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(max(3, args.warmup)):
+    warm = max(3, args.warmup)
+    for _ in range(warm):
         step()
-    stage = [new_events(4) for _ in range(args.steps)]
-    t_begin, t_end = new_events(2)
-    barrier()
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(ctx.local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    t_begin.record()
-    for i in range(args.steps):
-        step(stage[i])
-    t_end.record()
-    barrier()
-    total_ms = t_begin.elapsed_time(t_end)
+    total_ms, stage = timed_steps(args.steps)
     clocks = sampler.stop() if rank == 0 else None
     tokens = L * w.T
     ms_per_step, value = aggregate_replicas(total_ms, args.steps, tokens, dist, dev)
 
-    k1 = sum(ev[0].elapsed_time(ev[1]) for ev in stage) / args.steps
+    clear = sum(ev[0].elapsed_time(ev[1]) for ev in stage) / args.steps
+    k1 = sum(ev[1].elapsed_time(ev[2]) for ev in stage) / args.steps
     k3 = sum(ev[2].elapsed_time(ev[3]) for ev in stage) / args.steps
     peak, peak_kind = measured_peak_hbm()
     bytes_per_launch = algorithmic_bytes_per_token(w) * tokens
@@ -314,15 +355,17 @@ def run_gpu(args, w):
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "accumulate": "f32 (logits, scores and weights in f32; ids, loads, dispatch in int32)",
+        "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "accumulate": "f32 (logits, scores and weights in f32; ids, loads, dispatch in int32)",
         "data": "synthetic", "config": workload_config(w, L, n_copies),
         "roofline": {"bound": "hbm", "kernel": router_kernel_name(w, L),
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": recorded_traffic(w.name, tokens),
                      "bytes_per_launch": bytes_per_launch},
-        "path": {"router_select_ms": k1, "dispatch_ms": k3, "path_gbs": path_gbs,
-                 "path_frac_of_hbm_peak": path_gbs / peak, "path_frac_of_8tbs": path_gbs / 8000.0},
+        "path": {"flags_clear_ms": clear, "router_select_ms": k1, "dispatch_ms": k3,
+                 "path_gbs": path_gbs, "path_frac_of_hbm_peak": path_gbs / peak,
+                 "path_frac_of_8tbs": path_gbs / 8000.0},
         "routing": {"mean_imbalance_max_over_mean": imb, "I_agg": float(I_agg[0].item()),
                     "I_agg_bins": float(I_agg[1].item()),
                     "MV_max_over_layers": float(I_layers.max().item()) - 1.0,
@@ -336,11 +379,61 @@ def run_gpu(args, w):
         "clocks": clocks,
     }
 
+    plain = args.granularity == 1 and args.random_trim is None
+    if plain and world == 1:
+        # the same launch with every token on the top-k branch (eps_high = 0): what the router,
+        # the score epilogue and the bookkeeping of the selection cost when nothing is decided
+        n0 = max(3, min(args.steps, 8))
+        zero = [0.0] * L
+        for _ in range(2):
+            step(eps=zero)
+        _, st0 = timed_steps(n0, zero)
+        k1_0 = sum(ev[1].elapsed_time(ev[2]) for ev in st0) / n0
+        step()                       # leave the outputs of the rule itself behind
+        torch.cuda.synchronize()
+        result["selection"] = {
+            "router_select_ms_without_decisions": k1_0,
+            "kernel_ns_per_token_of_a_layer": k1 * 1e6 / w.T,
+            "budget_ns_per_token_at_70pct_of_hbm_peak":
+                bytes_per_launch / (0.7 * peak * 1e9) * 1e9 / w.T,
+            "note": "the ordered selection is one dependency chain per layer, all layers "
+                    "concurrent and overlapped with the router: kernel time / tokens of a layer "
+                    "bounds a chain step from above"}
+
     # end to end through the host-buffer entry point: H2D of the inputs, D2H of the results
-    if world == 1 or rank == 0:
+    if full and rank == 0:
         result["e2e"] = e2e_host(args, w, L, data, p, laser, torch, dev)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = cpu_baseline(args, w, L, data, np)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and plain:
+        base = cpu_baseline_and_agreement(args, w, L, data, np, torch, laser, synth, dev, full)
+        if full:
+            result["cpu_baseline"] = base.pop("cpu_baseline")
+        else:
+            result["cpu_oracle_sample"] = base.pop("cpu_baseline")
+        result["routing"].update(base.pop("routing"))
+        result["agreement"] = base.pop("agreement")
+        if "selection" in result:
+            nd = result["routing"]["decision_tokens_frac"] * w.T
+            result["selection"]["decision_tokens_per_layer"] = nd
+            if nd > 0:
+                result["selection"]["extra_ns_per_decision_token"] = \
+                    max(0.0, k1 - result["selection"]["router_select_ms_without_decisions"]) * 1e6 / nd
+    if full and rank == 0 and world == 1 and args.sustained_seconds > 0:
+        n = max(args.steps, int(args.sustained_seconds * 1e3 / ms_per_step) + 1)
+        sampler = ClockSampler(ctx.local)
+        sampler.start()
+        time.sleep(0.2)
+        e0, e1 = new_events(torch, 2)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n
+        result["sustained"] = {"steps": n, "seconds": ms * n * 1e-3, "ms_per_step": ms,
+                               "value": tokens / (ms * 1e-3),
+                               "path_frac_of_hbm_peak": bytes_per_launch / (ms * 1e-3) / 1e9 / peak,
+                               "clocks": sampler.stop()}
     if args.imbalance_batches > 0 and rank == 0:
         result["imbalance_study"] = imbalance_study(args, w, L, data, laser, synth, torch, dev,
                                                     loads, bins, ws)
@@ -352,11 +445,9 @@ def run_gpu(args, w):
         result["drift_from_the_rule"] = {
             "tokens_with_a_different_expert_set": float(1.0 - same.double().mean().item()),
             "mean_imbalance_of_the_rule": exact_imb, "mean_imbalance_of_this_variant": imb}
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
-    if rank == 0:
-        print(json.dumps(result))
+    del data, hiddens, out, ws, state
+    torch.cuda.empty_cache()
+    return result
 
 
 def imbalance_study(args, w, L, data, laser, synth, torch, dev, loads, bins, ws):
@@ -449,18 +540,17 @@ def score_stats_report(args, w, L, data, p, laser, torch, loads, bins, ws):
             "note": "one call (memset and two kernels) on logits just written, so partly in L2"}
 
 
-def run_decode(args, w):
+def run_decode(args, w, ctx, full):
     """Decode stream: `S` successive calls of T tokens each, same W_g, load state carried
     from call to call.  One bench step = one pass over the whole stream, replayed as a CUDA
-    graph; plain stream launches are timed beside it."""
+    graph; plain stream launches are timed beside it, then every call on its own (launch to
+    completion) for the latency distribution, next to the same figures for an empty kernel."""
     import numpy as np
     import torch
 
     from paper_2510_03293_b200 import laser, synth
 
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
+    dev = ctx.dev
     S = args.decode_steps or w.layers
     data = synth.make_workload_torch(w, dev, seed=args.seed, layers=S)
     hidden = data["hidden"]                      # [S, T, d]: call s routes hidden[s]
@@ -476,14 +566,17 @@ def run_decode(args, w):
         torch.empty((S, w.T * w.k), dtype=torch.int32, device=dev),
         loads, bins, None, torch.zeros((1,), dtype=torch.int32, device=dev))
 
+    def one_call(s_):
+        o = laser.RouteResult(outs.expert_ids[s_:s_ + 1], outs.weights[s_:s_ + 1],
+                              outs.offsets[s_:s_ + 1], outs.perm[s_:s_ + 1], loads, bins, None,
+                              outs.status)
+        laser.route_layers(hidden[s_:s_ + 1], wg, bias, loads, p, bin_loads=bins, out=o,
+                           workspace=ws)
+
     def one_pass():
         loads.zero_(); bins.zero_()
         for s_ in range(S):
-            o = laser.RouteResult(outs.expert_ids[s_:s_ + 1], outs.weights[s_:s_ + 1],
-                                  outs.offsets[s_:s_ + 1], outs.perm[s_:s_ + 1], loads, bins, None,
-                                  outs.status)
-            laser.route_layers(hidden[s_:s_ + 1], wg, bias, loads, p, bin_loads=bins, out=o,
-                               workspace=ws)
+            one_call(s_)
 
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
@@ -492,6 +585,12 @@ def run_decode(args, w):
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
             one_pass()
+        empty_graph = torch.cuda.CUDAGraph()
+        laser.test_launch_empty(side)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(empty_graph, stream=side):
+            for _ in range(S):
+                laser.test_launch_empty(side)
     torch.cuda.synchronize()
 
     def timed(fn, n):
@@ -504,9 +603,24 @@ def run_decode(args, w):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / n
 
+    def each_alone(fn, n):
+        """us from launch to completion of n calls made one at a time (the stream is idle
+        before each): what a decode loop that needs the result before its next step sees."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        us = []
+        for i in range(n):
+            torch.cuda.synchronize()
+            e0.record()
+            fn(i)
+            e1.record()
+            e1.synchronize()
+            us.append(e0.elapsed_time(e1) * 1e3)
+        return {"mean": sum(us) / len(us), "p50": percentile(us, 0.5), "p99": percentile(us, 0.99),
+                "calls": n}
+
     for _ in range(max(3, args.warmup)):
         graph.replay()
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(ctx.local)
     sampler.start(); time.sleep(0.3)
     ms_graph = timed(graph.replay, args.steps)
     clocks = sampler.stop()
@@ -514,6 +628,12 @@ def run_decode(args, w):
     ms_plain = timed(one_pass, max(1, min(args.steps, 3)))
     same = bool(torch.equal(ids_graph, outs.expert_ids) and torch.equal(loads_graph, loads))
     status = int(outs.status.item())
+    loads.zero_(); bins.zero_()
+    latency = each_alone(one_call, S)
+    floor_alone = each_alone(lambda i: laser.test_launch_empty(), min(S, 1024))
+    for _ in range(3):
+        empty_graph.replay()
+    floor_graph_us = timed(empty_graph.replay, max(3, min(args.steps, 10))) * 1e3 / S
 
     # end to end: every call copies its hidden states in and its results out
     h_hidden = hidden[:min(S, 256)].cpu().pin_memory()
@@ -535,7 +655,7 @@ def run_decode(args, w):
     tokens = S * w.T
     bytes_per_pass = algorithmic_bytes_per_token(w) * tokens
     gbs = bytes_per_pass / (ms_graph * 1e-3) / 1e9
-    print(json.dumps({
+    result = {
         "metric": METRIC, "value": tokens / (ms_graph * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_graph,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -546,17 +666,39 @@ def run_decode(args, w):
                    "cache": "every call reads its own %.2f MB of hidden states (%.2f GB per pass)"
                             % (2.0 * w.T * w.d / 1e6, 2.0 * tokens * w.d / 1e9)},
         "decode": {"us_per_call_graph": ms_graph * 1e3 / S, "us_per_call_stream_launches":
-                   ms_plain * 1e3 / S, "calls_per_pass": S, "graph_equals_stream_launches": same},
+                   ms_plain * 1e3 / S, "calls_per_pass": S, "graph_equals_stream_launches": same,
+                   "latency_us_one_call_at_a_time": latency,
+                   "launch_floor_us": {"empty_kernel_one_at_a_time": floor_alone,
+                                       "empty_kernel_per_graph_node": floor_graph_us},
+                   "graph_nodes_per_call": DECODE_NODES_PER_CALL},
         "roofline": {"bound": "hbm", "kernel": router_kernel_name(w, 1), "achieved": gbs,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": gbs / peak,
-                     "traffic": None, "bytes_per_launch": bytes_per_pass / S,
+                     "traffic": recorded_traffic(w.name, w.T), "bytes_per_launch": bytes_per_pass / S,
                      "note": "latency-bound: 0.26 MB per call"},
+        "path": {"path_gbs": gbs, "path_frac_of_hbm_peak": gbs / peak,
+                 "path_frac_of_8tbs": gbs / 8000.0},
         "routing": {"status_word": status},
         "gpu_launches": launches_per_step(w, 1) * S * args.steps, "clocks": clocks,
         "e2e": {"value": w.T / e2e_sec, "unit": UNIT, "ms_per_step": e2e_sec * 1e3 * S,
                 "us_per_call": e2e_sec * 1e6, "h2d_bytes_per_step": h2d * S,
                 "d2h_bytes_per_step": d2h * S, "calls_timed": int(h_hidden.shape[0])},
-    }))
+    }
+    if not args.no_cpu_baseline:
+        # the oracle on the concatenated stream (per-token load updates make one call over all
+        # the tokens equal to the sequence of calls), first 16384 tokens
+        n_calls = min(S, 16384 // w.T)
+        cat = {"hidden": hidden[:n_calls].reshape(1, n_calls * w.T, w.d), "w_g": wg, "bias": bias,
+               "eps_high": [w.eps_high[0]], "t_fix": [w.t_fix]}
+        wcat = dataclasses_replace(w, T=n_calls * w.T, layers=1)
+        base = cpu_baseline_and_agreement(args, wcat, 1, cat, np, torch, laser, synth, dev, False)
+        result["cpu_oracle_sample"] = base["cpu_baseline"]
+        result["routing"].update(base["routing"])
+        result["agreement"] = base["agreement"]
+        result["agreement"]["sample"] = ("the first %d calls as one call of %d tokens; " %
+                                         (n_calls, n_calls * w.T)) + "oracle on its own logits"
+    del data, hidden, outs, graph, empty_graph
+    torch.cuda.empty_cache()
+    return result
 
 
 def e2e_host(args, w, L, data, p, laser, torch, dev):
@@ -585,25 +727,164 @@ def e2e_host(args, w, L, data, p, laser, torch, dev):
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n}
 
 
-def cpu_baseline(args, w, L, data, np):
+def cpu_baseline_and_agreement(args, w, L, data, np, torch, laser, synth, dev, full):
+    """The CPU-baseline leg: the oracle as it stands, on the host cores, on a bounded sample of
+    the workload.  Its first sampled layer (the first 16384 tokens of it for longer layers) is
+    also compared with the GPU path: the oracle computes its OWN logits in fp64 from the same
+    bf16 inputs, so one token that falls on the other side of a threshold changes the loads seen
+    by every later token; reported are how many tokens still choose the same expert set, the
+    first token that differs, and the balance figures of both runs.  (The bit-exact comparison
+    given the GPU's fp32 logits is repeated here on the same sample.)"""
     import oracle
 
     oracle.build()
-    n_sample = min(L, args.ref_layers)
+    i16 = torch.int16
+    Ts = min(w.T, 16384)
+    n_sample = min(L, args.ref_layers) if full else 1
     layers_data = []
     for l in range(n_sample):
-        hb = data["hidden"][l].view(__import__("torch").int16).cpu().numpy().view(np.uint16)
-        wb = data["w_g"][l].view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+        hb = data["hidden"][l, :Ts].view(i16).cpu().numpy().view(np.uint16)
+        wb = data["w_g"][l].view(i16).cpu().numpy().view(np.uint16)
         layers_data.append((hb, wb, data["bias"][l].cpu().numpy()))
+    ws_ = dataclasses_replace(w, T=Ts)
+    e2b = synth.default_expert_to_bin(w.E, w.n_bins)
+    z, zb = np.zeros(w.E, np.int32), np.zeros(w.n_bins, np.int32)
+    eps0, tf0 = data["eps_high"][0], data["t_fix"][0]
+    # first pass, kept: the oracle's whole path on layer 0 with its own logits
+    t0 = time.perf_counter()
+    hb, wb, bias = layers_data[0]
+    ref = oracle.route_full(hb, wb, bias, z, e2b, zb, w.k, w.c, eps0, tf0, bool(w.renormalize))
+    first = time.perf_counter() - t0
     total, passes = 0.0, 0
-    while total < args.cpu_seconds and passes < 64:
-        total += oracle_pass(oracle, np, layers_data, w, data["eps_high"], data["t_fix"])
+    budget = args.cpu_seconds if full else 0.0
+    while total < budget and passes < 64:
+        total += oracle_pass(oracle, np, layers_data, ws_, data["eps_high"], data["t_fix"])
         passes += 1
+    if passes == 0:
+        total, passes, n_timed = first, 1, 1
+    else:
+        n_timed = n_sample
     sec = total / passes
-    return {"value": n_sample * w.T / sec, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
-            "kind": "oracle", "seconds": total,
-            "sample": "%d of %d layers (%d tokens) x %d passes, fp64 contraction with OpenMP over "
-                      "tokens, ordered scan on one core" % (n_sample, L, n_sample * w.T, passes)}
+    cores = len(os.sched_getaffinity(0))
+    base = {"value": n_timed * Ts / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "seconds": total,
+            "sample": "%d of %d layers%s (%d tokens) x %d passes, fp64 contraction with OpenMP over "
+                      "tokens, ordered scan on one core" %
+                      (n_timed, L, "" if Ts == w.T else ", first %d tokens of each" % Ts,
+                       n_timed * Ts, passes)}
+
+    # the GPU path on the same sample
+    p = laser.make_params(Ts, w.d, w.E, w.k, w.c, eps0, tf0, w.renormalize, w.n_bins)
+    loads = torch.zeros((1, w.E), dtype=torch.int32, device=dev)
+    r = laser.route_layers(data["hidden"][:1, :Ts].contiguous(), data["w_g"][:1], data["bias"][:1],
+                           loads, p, want_logits=True)
+    torch.cuda.synchronize()
+    ids_g = r.expert_ids[0].cpu().numpy()
+    x_g = r.logits[0].cpu().numpy()
+    cnt_g = np.diff(r.offsets[0].cpu().numpy()).astype(np.float64)
+    exact = oracle.route(x_g, z, w.k, w.c, eps0, tf0, bool(w.renormalize))
+    same = (np.sort(ids_g, 1) == np.sort(ref["expert_ids"], 1)).all(1)
+    differ = np.flatnonzero(~same)
+    cnt_o = ref["counts"].astype(np.float64)
+    imb = lambda c: float(c.max() / c.mean()) if c.sum() > 0 else 1.0
+    agreement = {
+        "sample": "layer 0, %d tokens; oracle on its own fp64-accumulated logits" % Ts,
+        "set_agreement_frac": float(same.mean()),
+        "first_divergent_token": int(differ[0]) if differ.size else None,
+        "logits_max_abs_err": float(np.max(np.abs(x_g - ref["logits"]))),
+        "imbalance_gpu": imb(cnt_g), "imbalance_oracle": imb(cnt_o),
+        "MV_gpu": imb(cnt_g) - 1.0, "MV_oracle": imb(cnt_o) - 1.0,
+        "bit_exact_given_gpu_logits": bool(np.array_equal(ids_g, exact[0]) and
+                                           np.array_equal(loads[0].cpu().numpy(), exact[2])),
+    }
+    # routing statistics of the sample (oracle run): expansion rule and final assignment
+    cs = ref["cstar"]
+    x = ref["logits"]
+    expanded = cs > 0
+    order = np.argsort(-x, axis=1, kind="stable")[:, :w.c]
+    sc = np.take_along_axis(oracle.softmax(x), order, 1)
+    thr = (np.float32(tf0) * sc[:, 0]).astype(np.float32)
+    m_prime = (sc >= thr[:, None]).sum(1)
+    topk = np.sort(oracle.topk(x, w.k), 1)
+    routing = {
+        "expanded_frac": float(expanded.mean()),
+        "mean_m_prime": float(m_prime[expanded].mean()) if expanded.any() else 0.0,
+        "mean_cstar": float(cs[expanded].mean()) if expanded.any() else 0.0,
+        "decision_tokens_frac": float((cs > w.k).mean()),
+        "differs_from_topk_frac": float((np.sort(ref["expert_ids"], 1) != topk).any(1).mean()),
+    }
+    return {"cpu_baseline": base, "agreement": agreement, "routing": routing}
+
+
+def dataclasses_replace(w, **kw):
+    import dataclasses
+
+    return dataclasses.replace(w, **kw)
+
+
+def one_core_oracle(name):
+    """The oracle's whole path on one workload layer with OpenMP held to one thread (a child
+    process, since the thread count is fixed when the library loads)."""
+    code = ("import sys, time, json, numpy as np; sys.path.insert(0, %r); import oracle; "
+            "from paper_2510_03293_b200 import synth; w = synth.WORKLOADS[%r]; "
+            "hb, wb, b = synth.make_workload_layer(w, 0); "
+            "e2b = synth.default_expert_to_bin(w.E, w.n_bins); "
+            "f = lambda: oracle.route_full(hb, wb, b, np.zeros(w.E, np.int32), e2b, "
+            "np.zeros(w.n_bins, np.int32), w.k, w.c, w.eps_for_layer(0), w.t_fix, bool(w.renormalize)); "
+            "f(); t = time.perf_counter(); f(); print(json.dumps(time.perf_counter() - t))" % (ROOT, name))
+    try:
+        out = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, OMP_NUM_THREADS="1"),
+                             capture_output=True, text=True, timeout=120)
+        sec = float(json.loads(out.stdout.strip().splitlines()[-1]))
+    except Exception as e:   # noqa: BLE001
+        return {"error": repr(e)}
+    from paper_2510_03293_b200 import synth
+
+    w = synth.WORKLOADS[name]
+    return {"value": w.T / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": sec,
+            "sample": "one layer of %d tokens, one pass" % w.T}
+
+
+def free_port():
+    import socket
+
+    with socket.socket() as s_:
+        s_.bind(("127.0.0.1", 0))
+        return s_.getsockname()[1]
+
+
+def spawn_replicas(n, argv):
+    """Starts n copies of this program, one per GPU, as the ranks of one job (the launch torchrun
+    would do) and returns the largest exit code.  Rank 0 prints the JSON line."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + argv, env=env))
+    return max(p_.wait() for p_ in procs)
+
+
+def selftest_replicas():
+    """CPU check of the replica plumbing (gloo): every rank reports a different time; the line
+    must carry the slowest one and the tokens of all ranks."""
+    import torch
+    import torch.distributed as dist
+
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms, value = aggregate_replicas(10.0 * (rank + 1), 5, 1000, dist, torch.device("cpu"))
+    dist.barrier()
+    dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"n_gpus": world, "ms_per_step": ms, "value": value}))
+
+
+SUB_WORKLOADS = ("tiny", "deepseek", "decode", "stress")
+# what a sub-workload's record keeps (the full records are printed by --workload NAME)
+SUB_KEYS = ("value", "unit", "ms_per_step", "steps", "config", "roofline", "path", "routing",
+            "selection", "agreement", "cpu_oracle_sample", "cpu_oracle_one_core", "decode",
+            "gpu_launches", "clocks")
 
 
 def main():
@@ -612,13 +893,17 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="laser", choices=["laser", "reference"])
-    ap.add_argument("--workload", default="mixtral")
+    ap.add_argument("--workload", default=None,
+                    help="one workload only (tiny, mixtral, deepseek, decode, stress); default: "
+                         "mixtral as the line's value with the other four under 'workloads'")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-layers", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0,
                     help="CPU work spent on the cpu_baseline leg")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the sustained loop of the headline step (0 = skip)")
     ap.add_argument("--decode-steps", type=int, default=None,
                     help="decode stream: successive 64-token calls per pass (default 4096)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -638,27 +923,45 @@ def main():
                     help="load-update granularity: 1 = the method's rule (default); 0 or a "
                          "multiple of 32 = the RELAXED variant, reported as such with its drift "
                          "from the rule")
+    ap.add_argument("--selftest-replicas", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))
+    if args.selftest_replicas:
+        return selftest_replicas()
 
     from paper_2510_03293_b200 import synth
 
-    w = synth.WORKLOADS[args.workload]
-    over = {}
-    if args.eps_high is not None:
-        over["eps_high"] = (args.eps_high,)
-    if args.t_fix is not None:
-        over["t_fix"] = args.t_fix
-    if args.c is not None:
-        over["c"] = args.c
-    if over:
-        import dataclasses
-        w = dataclasses.replace(w, **over)
+    def workload(name):
+        w = synth.WORKLOADS[name]
+        over = {}
+        if args.eps_high is not None:
+            over["eps_high"] = (args.eps_high,)
+        if args.t_fix is not None:
+            over["t_fix"] = args.t_fix
+        if args.c is not None:
+            over["c"] = args.c
+        return dataclasses_replace(w, **over) if over else w
+
+    headline = args.workload or "mixtral"
     if args.impl == "reference":
-        run_reference(args, w)
-    elif w.persistent_loads:
-        run_decode(args, w)
-    else:
-        run_gpu(args, w)
+        return run_reference(args, workload(headline))
+
+    ctx = Context()
+    run = lambda w, full: (run_decode if w.persistent_loads else run_layers)(args, w, ctx, full)
+    result = run(workload(headline), True)
+    if args.workload is None and ctx.world == 1 and args.layers is None:
+        subs = {}
+        for name in SUB_WORKLOADS:
+            r = run(workload(name), False)
+            if name == "tiny" and not args.no_cpu_baseline:
+                r["cpu_oracle_one_core"] = one_core_oracle(name)
+            subs[name] = {k_: r[k_] for k_ in SUB_KEYS if k_ in r}
+        result["workloads"] = subs
+    ctx.close()
+    if ctx.rank == 0:
+        print(json.dumps(result))
 
 
 if __name__ == "__main__":

@@ -36,6 +36,13 @@ int laser_test_set_router(int mode);
  */
 int laser_test_withhold_tile(int tile, long long wait_cycles);
 
+/*
+ * Enqueues one empty kernel (one block of 32 threads that does nothing) on cuda_stream (a
+ * cudaStream_t passed as void*), so that a benchmark can time the launch floor of this library's
+ * kernels on the machine at hand.  Returns 0, or -1 if the launch failed.
+ */
+int laser_test_launch_empty(void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

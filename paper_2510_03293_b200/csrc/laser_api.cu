@@ -182,6 +182,15 @@ extern "C" int laser_test_set_router(int mode) {
   return prev;
 }
 
+namespace {
+__global__ void k_empty() {}
+}  // namespace
+
+extern "C" int laser_test_launch_empty(void* cuda_stream) {
+  k_empty<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+}
+
 extern "C" int laser_test_withhold_tile(int tile, long long wait_cycles) {
   if (tile >= 0 && wait_cycles < 1) return -1;
   g_test_withhold_tile = tile < 0 ? -1 : tile;

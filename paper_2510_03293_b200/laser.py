@@ -39,7 +39,7 @@ EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_ro
            "laser_route_host", "laser_route_static", "laser_imbalance",
            "laser_score_stats")
 # include/laser_test_hooks.h: controls for the tests, not part of the routing interface
-TEST_EXPORTS = ("laser_test_set_router", "laser_test_withhold_tile")
+TEST_EXPORTS = ("laser_test_set_router", "laser_test_withhold_tile", "laser_test_launch_empty")
 
 
 class LaserParams(ctypes.Structure):
@@ -89,6 +89,8 @@ _lib.laser_test_set_router.argtypes = [ctypes.c_int]
 _lib.laser_test_set_router.restype = ctypes.c_int
 _lib.laser_test_withhold_tile.argtypes = [ctypes.c_int, ctypes.c_longlong]
 _lib.laser_test_withhold_tile.restype = ctypes.c_int
+_lib.laser_test_launch_empty.argtypes = [_vp]
+_lib.laser_test_launch_empty.restype = ctypes.c_int
 
 
 class LaserError(RuntimeError):
@@ -113,6 +115,16 @@ def test_withhold_tile(tile: int, wait_cycles: int = 0) -> None:
         raise ValueError("wait_cycles must be positive")
 
 
+def test_launch_empty(stream=None) -> None:
+    """laser_test_launch_empty: one empty kernel on the stream (launch-floor measurements)."""
+    import torch
+
+    s = torch.cuda.current_stream() if stream is None else stream
+    if int(_lib.laser_test_launch_empty(s.cuda_stream)) != 0:
+        raise LaserError(ERR_CUDA)
+
+
+test_launch_empty.__test__ = False
 test_set_router.__test__ = False          # not pytest cases, whatever the names suggest
 test_withhold_tile.__test__ = False
 

@@ -44,6 +44,26 @@ def test_two_replicas_take_the_slowest_time_and_add_their_tokens():
         assert abs(value - 2 * 1000 / 4.0e-3) < 1e-6     # tokens of both ranks over that time
 
 
+def test_bench_starts_its_own_replicas_when_not_under_torchrun():
+    """`bench.py --gpus 2` outside torchrun starts two ranks itself; here they run the CPU
+    self-test of the replica plumbing (gloo) instead of the GPU benchmark."""
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2",
+                          "--selftest-replicas"], env=env, capture_output=True, text=True,
+                         timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                               # rank 0 alone prints
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2
+    assert abs(rec["ms_per_step"] - 4.0) < 1e-9          # the slower rank's 20 ms over 5 steps
+    assert abs(rec["value"] - 2 * 1000 / 4.0e-3) < 1e-6
+
+
 def test_single_replica_needs_no_process_group():
     sys.path.insert(0, ROOT)
     import bench
