@@ -17,9 +17,12 @@ constexpr int kRouterWarps = kK2Threads / 32;
 template <int NT, int MT>
 __host__ __device__ constexpr int router_rows() { return kRouterWarps * MT * 16; }
 
-// logits tile of the block
-__host__ __device__ inline size_t router_smem_bytes(int NT, int MT) {
+// logits tile of the block, then one mask scratch of NT * 8 words per warp (see group_epilogue)
+__host__ __device__ inline size_t router_tile_bytes(int NT, int MT) {
   return sizeof(float) * kRouterWarps * MT * 16 * (NT * 8 + 1);
+}
+__host__ __device__ inline size_t router_smem_bytes(int NT, int MT) {
+  return router_tile_bytes(NT, MT) + (NT * 8 > 32 ? sizeof(uint32_t) * kRouterWarps * NT * 8 : 0);
 }
 
 template <int NT, int MT, int KU, int CMAX>
@@ -39,16 +42,18 @@ __global__ void __launch_bounds__(kK2Threads) k12_route_select(const RouteArgs A
   const int local_layer = b % n_layers;
   const int rt = b / n_layers;
   float* tiles = reinterpret_cast<float*>(dyn_smem);
+  uint32_t* fm = reinterpret_cast<uint32_t*>(dyn_smem + router_tile_bytes(NT, MT)) + warp * (NT * 8);
   const long long tok0 = (long long)rt * RR + (long long)warp * (MT * 16);
   if (tok0 < A.T) router_warp<NT, MT, KU>(A, local_layer, tok0, tiles + (size_t)warp * (MT * 16) * LDS, lane);
   if (MT == 2) {
     // a warp's 32 rows are one group: no block-wide hand-over needed
-    if (tok0 < A.T) group_epilogue(A, local_layer, tok0, tiles + (size_t)warp * 32 * LDS, LDS, lane);
+    if (tok0 < A.T)
+      group_epilogue(A, local_layer, tok0, tiles + (size_t)warp * 32 * LDS, LDS, lane, fm);
   } else {
     __syncthreads();
     const long long gtok0 = (long long)rt * RR + (long long)warp * 32;
     if (warp * 32 < RR && gtok0 < A.T)
-      group_epilogue(A, local_layer, gtok0, tiles + (size_t)warp * 32 * LDS, LDS, lane);
+      group_epilogue(A, local_layer, gtok0, tiles + (size_t)warp * 32 * LDS, LDS, lane, fm);
   }
   __syncthreads();
   if (tid == 0 && rt != A.withhold_tile) {

@@ -38,11 +38,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 //   otherwise c* = max(k, #{j < c : s_pi(j) >= t_fix * s_pi(0)}).
 // Writes the record (c*, ranked ids, ranked scores) for the load-aware scan and, for every
 // token, the top-k ids and weights (final for the top-k branch, overwritten otherwise).
+// fm (shared memory, may be null): per-expert masks of the token's group; a token without a
+// load-dependent choice (top-k branch or c* == k) sets its bit for each of its k best.
 __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int E, int k, int c,
                                                float eps_high, float t_fix, int renorm,
                                                uint16_t* cstar, uint8_t* cand_ids,
                                                float* cand_scores, int32_t* expert_ids,
-                                               float* weights) {
+                                               float* weights, uint32_t* fm = nullptr,
+                                               uint32_t bit = 0) {
   float xmax = x[0];
   for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, x[i]);
 
@@ -85,6 +88,8 @@ __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int 
   if (top_k_branch && renorm) {
     for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
   }
+  if (fm && (top_k_branch || mprime <= k))
+    for (int j = 0; j < k; ++j) atomicOr(&fm[cand_ids[j]], bit);   // (reads its own stores)
 }
 
 // ---- RANDOM trimming (Algorithm 1, mode RANDOM) ---------------------------------------------
@@ -118,7 +123,8 @@ static __device__ __noinline__ void token_epilogue_random(const float* row, int 
                                                    unsigned long long seed, int layer, long long t,
                                                    uint16_t* cstar, uint8_t* cand_ids,
                                                    float* cand_scores, int32_t* expert_ids,
-                                                   float* weights) {
+                                                   float* weights, uint32_t* fm = nullptr,
+                                                   uint32_t bit = 0) {
   float xmax = row[0];
   for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, row[i]);
   float a[8];
@@ -168,6 +174,8 @@ static __device__ __noinline__ void token_epilogue_random(const float* row, int 
     *cstar = 0;
     if (renorm)
       for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
+    if (fm)
+      for (int j = 0; j < k; ++j) atomicOr(&fm[cand_ids[j]], bit);
     return;
   }
   const int cs = c < m ? c : m;
@@ -195,6 +203,8 @@ static __device__ __noinline__ void token_epilogue_random(const float* row, int 
     cand_scores[j] = __fdiv_rn(exp32(__fsub_rn(row[e], xmax)), Z);
   }
   *cstar = (uint16_t)cs;
+  if (fm && cs <= k)   // a sample of exactly k experts leaves nothing to decide
+    for (int j = 0; j < k; ++j) atomicOr(&fm[cand_ids[j]], bit);
 }
 
 // ---- score epilogue with sorting networks (one thread per token) ---------------------------
@@ -250,7 +260,8 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
                                                       int c, float eps_high, float t_fix,
                                                       int renorm, uint16_t* cstar,
                                                       uint8_t* cand_ids, float* cand_scores,
-                                                      int32_t* expert_ids, float* weights) {
+                                                      int32_t* expert_ids, float* weights,
+                                                      uint32_t* fm = nullptr, uint32_t bit = 0) {
   constexpr uint32_t IDX = N - 1;
   constexpr int SH = N == 64 ? 6 : 7;
   static_assert(N == 64 || N == 128, "index bits");
@@ -318,7 +329,7 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
   }
   if (!exact) {
     token_epilogue(row, E, k, c, eps_high, t_fix, renorm, cstar, cand_ids, cand_scores, expert_ids,
-                   weights);
+                   weights, fm, bit);
     return;
   }
   float Mk = 0.0f, thr = 0.0f;
@@ -338,6 +349,11 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
   }
   const bool top_k_branch = (Mk >= eps_high);
   *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
+  if (fm && (top_k_branch || mprime <= k)) {
+#pragma unroll
+    for (int r = 0; r < CL; ++r)
+      if (r < k) atomicOr(&fm[IDX - (R[r] & IDX)], bit);
+  }
   float wv[CL];   // combine weights of the k best
 #pragma unroll
   for (int r = 0; r < CL; ++r) wv[r] = (top_k_branch && renorm) ? __fdiv_rn(sv[r], Mk) : sv[r];
@@ -393,7 +409,8 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
                                                       float eps_high, float t_fix, int renorm,
                                                       bool write, uint16_t* cstar,
                                                       uint8_t* cand_ids, float* cand_scores,
-                                                      int32_t* expert_ids, float* weights) {
+                                                      int32_t* expert_ids, float* weights,
+                                                      uint32_t* fm = nullptr, uint32_t bit = 0) {
   constexpr int EPL = N / 8;
   const float ninf = __int_as_float(0xff800000);
   float x[EPL];
@@ -454,6 +471,8 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
     *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
     if (top_k_branch && renorm)
       for (int q = 0; q < k; ++q) weights[q] = __fdiv_rn(weights[q], Mk);
+    if (fm && (top_k_branch || mprime <= k))
+      for (int q = 0; q < k; ++q) atomicOr(&fm[cand_ids[q]], bit);
     return;
   }
   // ranking: c rounds of "best remaining" (local scan, then a 3-step butterfly over the group);
@@ -527,6 +546,11 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
     }
   }
   if (j == 0) *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
+  if (fm && (top_k_branch || mprime <= k)) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (8 * q + j < k) atomicOr(&fm[ki[q]], bit);
+  }
 }
 
 // One warp contracts ROWS = MT*16 consecutive tokens [tok0, tok0 + ROWS) of one layer with W_g
@@ -656,25 +680,47 @@ __device__ __forceinline__ void router_warp(const RouteArgs& A, int layer, long 
 
 }
 
-// Score epilogue of up to 32 tokens [tok0, tok0 + 32) by one warp, lane = token.  rows: the
-// tokens' logits in shared memory, row stride lds floats.
+// Writes the masks of one group of 32 tokens (fm, shared memory, [E]) to the workspace; called by
+// a full warp after its lanes have set their bits.
+__device__ __forceinline__ void publish_group_masks(const RouteArgs& A, int abs_layer, long long tok0,
+                                                    const uint32_t* fm, int lane) {
+  __syncwarp();
+  uint32_t* out = reinterpret_cast<uint32_t*>(A.ws + (size_t)abs_layer * A.ws_ls + A.lay.fmask) +
+                  (size_t)(tok0 >> 5) * A.E;
+  for (int e = lane; e < A.E; e += 32) out[e] = fm[e];
+}
+
+// Score epilogue of up to 32 tokens [tok0, tok0 + 32) by one warp, lane = token; every lane of
+// the warp must call.  rows: the tokens' logits in shared memory, row stride lds floats.
+// fm: the warp's mask scratch in shared memory ([E] words; only used, and only needed, when
+// E > 32).
 __device__ __forceinline__ void group_epilogue(const RouteArgs& A, int layer, long long tok0,
-                                               const float* rows, int lds, int lane) {
+                                               const float* rows, int lds, int lane,
+                                               uint32_t* fm) {
+  const bool masks = A.E > 32;
+  if (masks) {
+    for (int e = lane; e < A.E; e += 32) fm[e] = 0;
+    __syncwarp();
+  } else {
+    fm = nullptr;
+  }
   const long long t = tok0 + lane;
-  if (t >= A.T) return;
-  unsigned char* ws = A.ws + (size_t)(A.layer0 + layer) * A.ws_ls;
-  const int k = A.k, c = A.c;
-  const size_t lt = (size_t)(A.layer0 + layer) * A.T + t;
-  uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
-  uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
-  float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
-  if (A.trim_random)
-    token_epilogue_random(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer],
-                          A.renorm, A.seed, A.layer0 + layer, t, cs_p, ids_p, sc_p,
-                          A.expert_ids + lt * k, A.weights + lt * k);
-  else
-    token_epilogue(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
-                   cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k);
+  if (t < A.T) {
+    unsigned char* ws = A.ws + (size_t)(A.layer0 + layer) * A.ws_ls;
+    const int k = A.k, c = A.c;
+    const size_t lt = (size_t)(A.layer0 + layer) * A.T + t;
+    uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
+    uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
+    float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
+    if (A.trim_random)
+      token_epilogue_random(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer],
+                            A.renorm, A.seed, A.layer0 + layer, t, cs_p, ids_p, sc_p,
+                            A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
+    else
+      token_epilogue(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
+                     cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
+  }
+  if (masks) publish_group_masks(A, A.layer0 + layer, tok0, fm, lane);
 }
 
 
@@ -683,7 +729,7 @@ __device__ __forceinline__ void group_epilogue(const RouteArgs& A, int layer, lo
 // the partial sums meet in shared memory in a fixed order, and warps 0..3 score 4 tokens each.
 // NT: 8-expert column tiles.  smem: router_splitk_smem_bytes(NT).
 __host__ __device__ inline size_t router_splitk_smem_bytes(int NT) {
-  return sizeof(float) * (8 * 16 * NT * 8 + 16 * (NT * 8 + 8));
+  return sizeof(float) * (8 * 16 * NT * 8 + 16 * (NT * 8 + 8)) + sizeof(uint32_t) * NT * 8;
 }
 
 template <int NT, int KU>
@@ -778,6 +824,10 @@ __device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int laye
   __syncthreads();
   // logits = ((p0 + p1) + ... + p7) + bias, clamped; tile rows are LDS floats apart
   float* tile = smem + 8 * 16 * EP;
+  // masks of the tile's tokens without a load-dependent choice (16 tokens: half a group)
+  uint32_t* fm = E > 32 ? reinterpret_cast<uint32_t*>(tile + 16 * LDS) : nullptr;
+  if (fm)
+    for (int e = tid; e < E; e += blockDim.x) fm[e] = 0;
   const float* bias = A.bias ? A.bias + (size_t)abs_layer * E : nullptr;
   const float big = 3.402823466e+38f;
   for (int idx = tid; idx < 16 * EP; idx += blockDim.x) {
@@ -808,7 +858,7 @@ __device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int laye
                             reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
                             ws + A.lay.cand_ids + (size_t)t * c,
                             reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
-                            A.expert_ids + lt * k, A.weights + lt * k);
+                            A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << tid);
     }
   } else if (warp < 4) {
     const int r = warp * 4 + (lane >> 3);
@@ -823,7 +873,16 @@ __device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int laye
                               reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + tc,
                               ws + A.lay.cand_ids + (size_t)tc * c,
                               reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)tc * c,
-                              A.expert_ids + lt * k, A.weights + lt * k);
+                              A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << r);
+  }
+  if (fm) {
+    __syncthreads();
+    // this tile's 16-bit half of the group's mask words
+    uint16_t* out = reinterpret_cast<uint16_t*>(A.ws + (size_t)abs_layer * A.ws_ls + A.lay.fmask) +
+                    ((size_t)(rt >> 1) * E) * 2 + (rt & 1);
+    for (int e = tid; e < E; e += blockDim.x) out[2 * e] = (uint16_t)fm[e];
+    if ((rt & 1) == 0 && tok0 + 16 >= T)   // the group's upper half has no tokens: zero it
+      for (int e = tid; e < E; e += blockDim.x) out[2 * e + 1] = 0;
   }
 }
 

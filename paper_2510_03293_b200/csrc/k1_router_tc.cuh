@@ -146,6 +146,7 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
   constexpr int TMEM_COLS = N <= 32 ? 32 : (N <= 64 ? 64 : (N <= 128 ? 128 : 256));
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
+  __shared__ uint32_t s_fm[4 * N];   // masks of the tile's four groups (see group_epilogue)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = A.T, E = A.E, d = A.d;
   const int abs_layer = A.layer0 + layer;
@@ -248,6 +249,7 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
     const int k = A.k, c = A.c;
     unsigned char* ws = A.ws + (size_t)abs_layer * A.ws_ls;
     float* tile = reinterpret_cast<float*>(stages);
+    for (int i = tid; i < 4 * N; i += blockDim.x) s_fm[i] = 0;   // (a block barrier follows)
     if constexpr (N <= 128) {
       // N <= 128: all 128 rows of N + 1 floats (odd stride: a thread per row is conflict-free),
       // then warps 0..3 score one token per thread with sorting networks
@@ -281,6 +283,7 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
         }
       }
       const long long t = tok0 + tid;
+      uint32_t* fm = s_fm + warp * N;   // warps 0..3 each score one group of 32 tokens
       if (tid < kTcTileM && t < T) {
         const size_t lt = (size_t)abs_layer * T + t;
         uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
@@ -289,15 +292,18 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
         if (A.trim_random)
           token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
                                 A.t_fix[layer], A.renorm, A.seed, abs_layer, t, cs_p, ids_p, sc_p,
-                                A.expert_ids + lt * k, A.weights + lt * k);
+                                A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
         else if (c <= CL)
           token_epilogue_sorted<N, CL>(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
                                        A.t_fix[layer], A.renorm, cs_p, ids_p, sc_p,
-                                       A.expert_ids + lt * k, A.weights + lt * k);
+                                       A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
         else
           token_epilogue(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer],
-                         A.renorm, cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k);
+                         A.renorm, cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k,
+                         fm, 1u << lane);
       }
+      if (warp < 4 && tok0 + warp * 32 < T)
+        publish_group_masks(A, abs_layer, tok0 + warp * 32, fm, lane);
     } else {
     // N = 256: ROWS rows of N + 8 floats (the padding keeps the four 8-lane groups of a warp on
     // different banks), the 128 tokens in two passes of 64; 8 lanes score one token.
@@ -341,7 +347,8 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
                                 reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
                                 ws + A.lay.cand_ids + (size_t)t * c,
                                 reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
-                                A.expert_ids + lt * k, A.weights + lt * k);
+                                A.expert_ids + lt * k, A.weights + lt * k,
+                                s_fm + ((row0 + tid) >> 5) * N, 1u << (tid & 31));
         }
       }
       // groups of 8 lanes score one token each, 4 tokens per warp at a time
@@ -358,10 +365,14 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
                                  reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + tc,
                                  ws + A.lay.cand_ids + (size_t)tc * c,
                                  reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)tc * c,
-                                 A.expert_ids + lt * k, A.weights + lt * k);
+                                 A.expert_ids + lt * k, A.weights + lt * k,
+                                 s_fm + ((row0 + r) >> 5) * N, 1u << (r & 31));
       }
       __syncthreads();   // the tile is reused by the next pass
     }
+    // the masks of the tile's groups (every warp has passed the barrier above)
+    if (warp < 4 && (long long)rt * kTcTileM + warp * 32 < T)
+      publish_group_masks(A, abs_layer, (long long)rt * kTcTileM + warp * 32, s_fm + warp * N, lane);
   }
     }
   tc_fence_before();

@@ -31,6 +31,7 @@
 // device-bin sums.
 #pragma once
 #include "laser_common.cuh"
+#include "k2_chain.cuh"
 #include "k3_dispatch.cuh"
 
 namespace laser {
@@ -40,8 +41,6 @@ constexpr int kK2Warps = kK2Threads / 32;
 constexpr int kK2Batch = kK2Threads;     // tokens per batch, thread = token
 constexpr int kK2FastMaxLoad = 1 << 25;  // 32-bit keys (load << 5 | rank) stay below 2^31
 constexpr int kK2MaxSweeps = kK2Batch + 2;
-constexpr int kK2ChainMax = kK2Batch;    // E > 32, the rule's own order: batches with this many
-                                         // decision tokens or fewer take them one after the other
 constexpr long long kK2WaitCycles = 4000000000LL;  // default limit of a wait: ~2 s
 
 __host__ __device__ inline bool k2_fast_shape(int k, int c) { return c <= 32 && k <= 32; }
@@ -50,21 +49,21 @@ __host__ __device__ inline size_t k2_batch_bytes(int c) {
 }
 
 // Shared memory of the selection role:
-//   int32 L[E] | int32 Lin[E] | uint64 keys[c] | int32 wtot[8][max(E,32)] |
-//   uint32 mask[8][E] | int32 excl[8][E] (E > 32) | uint8 chosen[256][32] (E > 32) |
-//   chain mode (E > 32): int32 dexcl[8][E] | int32 dcnt[E] | lists | uint32 dseen[256][CMAX] |
-//   uint8 dcand[256][CMAX] | 2 batch buffers (c*, candidate ids)
+//   int32 L[E] | int32 Lin[E] | int32 Lvis[E] | uint64 keys[c] | int32 wtot[8][max(E,32)] |
+//   then either the batch fixed point's part
+//     uint32 mask[8][E] | int32 excl[8][E] | uint8 chosen[256][32] (all three E > 32 only) |
+//     2 batch buffers (c*, candidate ids)
+//   or (E > 32, the rule's own update order) the pipeline's part, k2_chain_smem_bytes()
 __host__ __device__ inline size_t k2_smem_bytes(int E, int c, int k) {
   const size_t Ew = E > 32 ? E : 32;
-  size_t b = 3 * align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c) +
-             align256(sizeof(int32_t) * kK2Warps * Ew);
+  const size_t b = 3 * align256(sizeof(int32_t) * E) + align256(sizeof(unsigned long long) * c) +
+                   align256(sizeof(int32_t) * kK2Warps * Ew);
   if (!k2_fast_shape(k, c)) return b;
-  if (E > 32) {
-    const size_t cmax = c <= 4 ? 4 : (c <= 8 ? 8 : (c <= 16 ? 16 : 32));   // the sorting width
-    b += 3 * align256(sizeof(int32_t) * kK2Warps * E) + align256(sizeof(int32_t) * E) +
-         (size_t)kK2Batch * 32 + 512 + (size_t)kK2Batch * cmax * 5;
-  }
-  return b + 2 * k2_batch_bytes(c);
+  size_t sweeps = 2 * k2_batch_bytes(c);
+  if (E <= 32) return b + sweeps;
+  sweeps += 2 * align256(sizeof(int32_t) * kK2Warps * E) + (size_t)kK2Batch * 32;
+  const size_t chain = k2_chain_smem_bytes(E, c);
+  return b + (sweeps > chain ? sweeps : chain);
 }
 
 // Calls of at most this many 32-token groups have their dispatch done by the selection block
@@ -94,7 +93,7 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 // Bounded: gives up after `limit` cycles and returns false; also false as soon as one of the
 // tiles reports that it gave up itself (flag < 0).  block = false only tests once.
 __device__ __forceinline__ bool k2_wait_ready(const int* ready, int router_rows, int t_first,
-                                              int t_last, long long limit, bool block = true) {
+                                              int t_last, long long limit, bool block) {
   const int lane = threadIdx.x & 31;
   const int rt0 = t_first / router_rows, rt1 = t_last / router_rows;
   const long long start = clock64();
@@ -142,13 +141,6 @@ struct K2Smem {
   uint32_t* mask;    // [8][E]  E > 32: bit i = token i of the warp chose this expert
   int32_t* excl;     // [8][E]  E > 32: exclusive prefix of the mask popcounts over warps
   uint8_t* chosen;   // [256][32] E > 32: current choice of every token, key order
-  int32_t* dexcl;    // [8][E]  E > 32, chain mode: decisions of each warp's tokens per expert
-  int32_t* dcnt;     // [E]     E > 32, chain mode: decisions so far in the batch per expert
-  uint8_t* dlist;    // [256]   E > 32, chain mode: the batch's decision tokens in order
-  int32_t* dwarp;    // [8]     E > 32, chain mode: decision tokens per warp
-  uint32_t* dseen;   // [256][CMAX] E > 32, chain mode: per decision token and candidate the load
-                     //         seen without the batch's decisions (all ones: no candidate)
-  uint8_t* dcand;    // [256][CMAX] E > 32, chain mode: the candidates' experts
 };
 
 // One batch of up to 256 tokens, thread = token, run by the whole block.
@@ -257,117 +249,6 @@ __device__ __forceinline__ void k2_batch(const K2Smem& sm, const uint16_t* cs_s,
   uint32_t* mk = sm.mask + warp * E;
   uint8_t* ch = sm.chosen + tid * 32;
 
-  // The rule's own order (strict) with decision tokens in the batch: the other tokens' increments
-  // are counted in parallel, every decision token works out in parallel the load each of its
-  // candidates would see without the decisions of this batch, and warp 0 then takes the decision
-  // tokens one after the other, lane = candidate: add the decisions so far for the candidate's
-  // expert, rank the keys with shuffles, the k smallest are the choice.  One step costs a
-  // shared-memory round trip and CMAX shuffles whatever the batch looks like, where the
-  // block-wide fixed point needs a sweep per link of the longest dependency chain.
-  if (strict && any_dec && n_dec <= kK2ChainMax) {
-    if (valid && !dec)
-      for (int j = 0; j < k; ++j) atomicOr(&mk[my[j]], 1u << lane);
-    const unsigned dmask = __ballot_sync(0xffffffffu, dec);
-    if (lane == 0) sm.dwarp[warp] = __popc(dmask);
-    for (int e = tid; e < E; e += kK2Threads) sm.dcnt[e] = 0;
-    for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.dexcl[i] = 0;
-    __syncthreads();   // masks of the fixed tokens and the warps' decision counts are complete
-    int at = 0;        // position of this decision token among the batch's decision tokens
-    if (dec) {
-      at = __popc(dmask & below);
-      for (int w = 0; w < warp; ++w) at += sm.dwarp[w];
-      sm.dlist[at] = (uint8_t)tid;
-    }
-    for (int e = tid; e < E; e += kK2Threads) {
-      int32_t run = 0;
-#pragma unroll
-      for (int w = 0; w < kK2Warps; ++w) {
-        sm.excl[w * E + e] = run;
-        run += __popc(sm.mask[w * E + e]);
-      }
-      sm.wtot[e] = run;
-    }
-    __syncthreads();   // excl is complete
-    // With a handful of decision tokens warp 0 lists their candidates itself and writes their
-    // results itself, which saves two block barriers; otherwise every decision token does.
-    const bool few = n_dec * CMAX <= 64;
-    if (!few) {
-      if (dec) {
-#pragma unroll
-        for (int r = 0; r < CMAX; ++r) {
-          const bool has = r < cs;
-          const int e = has ? (int)my[r] : 0;
-          sm.dseen[at * CMAX + r] =
-              has ? (uint32_t)(sm.L[e] + sm.excl[warp * E + e] + __popc(mk[e] & below))
-                  : 0xffffffffu;
-          sm.dcand[at * CMAX + r] = (uint8_t)e;
-        }
-      }
-      __syncthreads();   // every decision token's candidates and base loads are listed
-    }
-    uint8_t* dch = sm.chosen;   // [n_dec][k] chosen ranks in the order the method lists them
-    if (warp == 0) {
-      if (few) {
-        for (int it = lane; it < n_dec * CMAX; it += 32) {
-          const int i = it / CMAX, r = it - i * CMAX;
-          const int t = sm.dlist[i], w = t >> 5;
-          const bool has = r < (int)cs_s[t];
-          const int e = has ? (int)ids_s[t * c + r] : 0;
-          sm.dseen[it] = has ? (uint32_t)(sm.L[e] + sm.excl[w * E + e] +
-                                          __popc(sm.mask[w * E + e] & ((1u << (t & 31)) - 1)))
-                             : 0xffffffffu;
-          sm.dcand[it] = (uint8_t)e;
-        }
-        __syncwarp();
-      }
-      const bool mine = lane < CMAX;
-      uint32_t s_n = mine ? sm.dseen[lane] : 0xffffffffu;
-      int e_n = mine ? (int)sm.dcand[lane] : 0;
-      for (int i = 0; i < n_dec; ++i) {
-        const uint32_t s_i = s_n;
-        const int e = e_n;
-        if (mine && i + 1 < n_dec) {
-          s_n = sm.dseen[(i + 1) * CMAX + lane];
-          e_n = (int)sm.dcand[(i + 1) * CMAX + lane];
-        }
-        const bool has = s_i != 0xffffffffu;
-        const uint32_t key = has ? (((s_i + (uint32_t)sm.dcnt[e]) << 5) | (uint32_t)lane)
-                                 : 0xffffffffu;
-        int cnt = 0;
-#pragma unroll
-        for (int j = 0; j < CMAX; ++j) cnt += __shfl_sync(0xffffffffu, key, j) < key ? 1 : 0;
-        if (has && cnt < k) {
-          sm.dcnt[e] += 1;   // the candidates of one token are distinct experts
-          dch[i * k + cnt] = (uint8_t)lane;
-        }
-        __syncwarp();
-      }
-    }
-    if (!few) __syncthreads();   // dcnt and the chosen ranks are final
-    // chosen ranks out; dexcl[w][e] counts the decisions of warp w's tokens for expert e
-    if (!few || warp == 0) {
-      const int first = few ? lane : tid, step = few ? 32 : kK2Threads;
-      for (int idx = first; idx < n_dec * k; idx += step) {
-        const int i = idx / k, j = idx - i * k;
-        const int t = sm.dlist[i], r = dch[idx];
-        sel[t * k + j] = (uint8_t)r;
-        atomicAdd(&sm.dexcl[(t >> 5) * E + sm.dcand[i * CMAX + r]], 1);
-      }
-    }
-    __syncthreads();
-    for (int i = tid; i < kK2Warps * E; i += kK2Threads) {
-      const int w = i / E, e = i - w * E;
-      if (w * 32 < n_here) {
-        int32_t before = sm.excl[i];   // fixed tokens, then decisions, of the warps before w
-        for (int w2 = 0; w2 < w; ++w2) before += sm.dexcl[w2 * E + e];
-        g_base[i] = sm.L[e] - sm.Lin[e] + before;
-      }
-    }
-    __syncthreads();   // every thread has read the masks, excl, dexcl and sm.L of this batch
-    for (int e = tid; e < E; e += kK2Threads) sm.L[e] += sm.wtot[e] + sm.dcnt[e];
-    for (int i = tid; i < kK2Warps * E; i += kK2Threads) sm.mask[i] = 0;
-    return;
-  }
   if (valid)   // every token takes its k best to start with
     for (int j = 0; j < k; ++j) {
       ch[j] = my[j];
@@ -506,18 +387,12 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   sm.keys = reinterpret_cast<unsigned long long*>(p);  p += align256(sizeof(unsigned long long) * c);
   sm.wtot = reinterpret_cast<int32_t*>(p);    p += align256(sizeof(int32_t) * kK2Warps * Ew);
   sm.mask = nullptr; sm.excl = nullptr; sm.chosen = nullptr;
-  sm.dexcl = nullptr; sm.dcnt = nullptr; sm.dlist = nullptr; sm.dwarp = nullptr;
-  sm.dseen = nullptr; sm.dcand = nullptr;
-  if (E > 32 && k2_fast_shape(k, c)) {
+  unsigned char* chain_smem = p;   // E > 32 under the rule's own order: the pipeline's part
+  const bool chain = E > 32 && A.G == 1 && k2_fast_shape(k, c);
+  if (E > 32 && k2_fast_shape(k, c) && !chain) {
     sm.mask = reinterpret_cast<uint32_t*>(p);  p += align256(sizeof(int32_t) * kK2Warps * E);
     sm.excl = reinterpret_cast<int32_t*>(p);   p += align256(sizeof(int32_t) * kK2Warps * E);
     sm.chosen = p;                              p += (size_t)kK2Batch * 32;
-    sm.dexcl = reinterpret_cast<int32_t*>(p);  p += align256(sizeof(int32_t) * kK2Warps * E);
-    sm.dcnt = reinterpret_cast<int32_t*>(p);   p += align256(sizeof(int32_t) * E);
-    sm.dlist = p;                               p += 256;
-    sm.dwarp = reinterpret_cast<int32_t*>(p);  p += 256;
-    sm.dseen = reinterpret_cast<uint32_t*>(p); p += (size_t)kK2Batch * CMAX * sizeof(uint32_t);
-    sm.dcand = p;                               p += (size_t)kK2Batch * CMAX;
   }
   unsigned char* bufs = p;
   const size_t buf_bytes = k2_batch_bytes(c);
@@ -576,6 +451,10 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       }
       if (!ok && lane == 0) give_up();
     }
+  } else if (!SMALL && chain) {
+    if (tid == 0 && ready) const_cast<int*>(ready)[mode_word_index(T)] = 1;   // choices as masks
+    k2_chain_layer<CMAX>(A, layer, chain_smem, sm.L, sm.Lin, &s_gave_up, ready, router_rows,
+                         give_up);
   } else {
     const int n_batches = (T + kK2Batch - 1) / kK2Batch;
     // copies the c* and candidate ids of batch b into buffer b & 1 (cp.async, not waited for)

@@ -10,7 +10,9 @@
 // mask of its tokens sent there (the second term is then a population count), then every lane
 // finishes its own token:
 //   top-k branch (c* = 0): slots in score order; ids and weights were written by the router.
-//   c* > k: slots as the load-aware scan listed them (ascending load, then score rank).
+//   c* > k: slots as the load-aware scan listed them (ascending load, then score rank); where
+//           the scan left the choice as a bit mask over score ranks (the layer's mode word is
+//           set), the slot order is rebuilt like that of c* == k.
 //   c* == k: the set is the k best; slots ordered by (load seen, score rank), where the load
 //            seen by rank j is L_in[e] + its position inside e's segment.
 // w_j = s[expert of slot j], divided by the left-to-right sum over the slots if renormalising.
@@ -52,6 +54,8 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
   const uint8_t* cand = ws + A.lay.cand_ids + (size_t)t * c;
   const uint8_t* sel = ws + A.lay.sel_rank + (size_t)t * k;
   const int32_t* gb = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) + (size_t)g * E;
+  const bool as_masks =
+      reinterpret_cast<const int*>(ws + A.lay.ready)[mode_word_index(T)] != 0;
 
   for (int e = lane; e < E; e += 32) { base[e] = gb[e]; mask[e] = 0; }
   __syncwarp();
@@ -59,10 +63,15 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
 #pragma unroll
   for (int j = 0; j < KR; ++j) { ex[j] = 0; rk[j] = j; }
   if (valid) {
+    uint32_t chosen = (cs > k && as_masks)
+                          ? reinterpret_cast<const uint32_t*>(ws + A.lay.sel_mask)[t] : 0u;
 #pragma unroll
     for (int j = 0; j < KR; ++j)
       if (j < k) {
-        if (cs > k) rk[j] = sel[j];
+        if (cs > k) {
+          if (as_masks) { rk[j] = __ffs(chosen) - 1; chosen &= chosen - 1; }   // ascending rank
+          else rk[j] = sel[j];
+        }
         ex[j] = cand[rk[j]];
         atomicOr(&mask[ex[j]], 1u << lane);
       }
@@ -90,12 +99,13 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
   int slot[KR];
 #pragma unroll
   for (int j = 0; j < KR; ++j) { v[j] = 0.0f; slot[j] = j; }
-  if (cs > k) {
+  if (cs > k && !as_masks) {
 #pragma unroll
     for (int j = 0; j < KR; ++j)
       if (j < k) v[j] = sc[rk[j]];
   } else {
-    // c* == k: slots by (load seen, score rank); the load seen by rank j is L_in[e] + position
+    // the set is known, in ascending score rank (c* == k: the k best): slots by (load seen,
+    // score rank); the load seen by the expert of rank j is L_in[e] + position
     // (relaxed variant: + the assignments made before the token's chunk instead)
     const int32_t* gb0 = nullptr;
     if (A.G != 1)
@@ -106,7 +116,7 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
 #pragma unroll
     for (int j = 0; j < KR; ++j) {
       seen[j] = j < k ? lin_s[ex[j]] + (gb0 ? gb0[ex[j]] : pos[j]) : 0;
-      sj[j] = j < k ? sc[j] : 0.0f;
+      sj[j] = j < k ? sc[rk[j]] : 0.0f;
     }
 #pragma unroll
     for (int j = 0; j < KR; ++j) {
@@ -162,6 +172,15 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
   const uint8_t* cand = ws + A.lay.cand_ids + (size_t)t * c;
   const uint8_t* sel = ws + A.lay.sel_rank + (size_t)t * k;
   const int32_t* gb = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) + (size_t)g * E;
+  const bool as_masks =
+      reinterpret_cast<const int*>(ws + A.lay.ready)[mode_word_index(T)] != 0;
+  const uint32_t chosen = (valid && cs > k && as_masks)
+                              ? reinterpret_cast<const uint32_t*>(ws + A.lay.sel_mask)[t] : 0u;
+  // candidate rank of slot j as the selection left it (masks: ascending score rank)
+  auto rank_of = [&](int j) -> int {
+    if (cs <= k) return j;
+    return as_masks ? (int)__fns(chosen, 0, j + 1) : (int)sel[j];
+  };
 
   for (int e = lane; e < E; e += 32) { base[e] = gb[e]; mask[e] = 0; }
   __syncwarp();
@@ -170,7 +189,7 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
   // the number of earlier tokens of the group in that mask.
   if (valid)
     for (int j = 0; j < k; ++j) {
-      const uint8_t e = cand[cs > k ? sel[j] : j];
+      const uint8_t e = cand[rank_of(j)];
       pe[lane * k + j] = e;
       atomicOr(&mask[e], 1u << lane);
     }
@@ -196,7 +215,7 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
     return;
   }
   float sum = 0.0f;
-  if (cs > k) {
+  if (cs > k && !as_masks) {
     for (int j = 0; j < k; ++j) {
       const int e = mype[j];
       ids[j] = e;
@@ -226,7 +245,7 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
         slot += (Li < Lj || (Li == Lj && i < j)) ? 1 : 0;
       }
       ids[slot] = ej;
-      w[slot] = sc[j];
+      w[slot] = sc[rank_of(j)];
       perm[off[ej] + mypos[j]] = pair0 + slot;
     }
     if (A.renorm) {

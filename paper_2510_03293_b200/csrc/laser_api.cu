@@ -148,7 +148,7 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   }
   // clear the router's ready flags of these layers (one strided memset), then one launch for
   // the router and the ordered selection, one for the dispatch
-  const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 15) / 16 + 1);
+  const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 15) / 16 + 2);
   if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
                         (size_t)n, s) != cudaSuccess)
     return LASER_ERR_CUDA;

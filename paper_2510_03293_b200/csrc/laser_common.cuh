@@ -16,10 +16,18 @@ struct WorkspaceLayout {
   size_t sel_rank;     // uint8  [T, k]     rank positions chosen by the load-aware scan
   size_t grp_base;     // int32  [n_groups, E]  per-expert count of this call's assignments made
                        //                   before the group (load at group start minus L_in)
-  size_t ready;        // int32  [ceil(T/16)+1] router tiles published to the selection role
+  size_t fmask;        // uint32 [n_groups, E]  (E > 32 only) bit i: token i of the group has no
+                       //                   load-dependent choice and goes to this expert; router
+                       //                   tiles of 16 tokens write their 16-bit half
+  size_t sel_mask;     // uint32 [T]  (E > 32 only) the chosen candidates of a decision token as a
+                       //                   bit mask over score ranks, where the selection ran as
+                       //                   the pipeline of k2_chain.cuh (mode word = 1)
+  size_t ready;        // int32  [ceil(T/16)+2] router tiles published to the selection role
                        //                   (1 = records written, -1 = the tile gave up); the last
                        //                   word is the layer's abort word: non-zero once a wait ran
-                       //                   out, and then no later stage reads the layer's scratch
+                       //                   out, and then no later stage reads the layer's scratch;
+                       //                   the word after it is the mode word: 1 if the decision
+                       //                   tokens' choices are in sel_mask, 0 if in sel_rank
   size_t total;        // bytes per layer, multiple of 256
   int n_groups;        // ceil(T / 32): the ordered selection and the dispatch work on groups
                        // of 32 consecutive tokens
@@ -36,7 +44,9 @@ inline WorkspaceLayout make_layout(int T, int E, int k, int c) {
   w.cand_scores = off;  off = align256(off + sizeof(float) * (size_t)T * c);
   w.sel_rank = off;     off = align256(off + (size_t)T * k);
   w.grp_base = off;     off = align256(off + sizeof(int32_t) * (size_t)w.n_groups * E);
-  w.ready = off;        off = align256(off + sizeof(int32_t) * (size_t)((T + 15) / 16 + 1));
+  w.fmask = off;        off = align256(off + (E > 32 ? sizeof(uint32_t) * (size_t)w.n_groups * E : 0));
+  w.sel_mask = off;     off = align256(off + (E > 32 ? sizeof(uint32_t) * (size_t)T : 0));
+  w.ready = off;        off = align256(off + sizeof(int32_t) * (size_t)((T + 15) / 16 + 2));
   w.total = off;
   return w;
 }
@@ -75,6 +85,7 @@ struct RouteArgs {
 
 // The layer's abort word (see WorkspaceLayout::ready).
 __host__ __device__ inline size_t abort_word_index(int T) { return (size_t)((T + 15) / 16); }
+__host__ __device__ inline size_t mode_word_index(int T) { return abort_word_index(T) + 1; }
 
 // Rank position (in the score ranking) of slot j of token t as the selection left it:
 // tokens with c* > k were decided by the load-aware scan (sel_rank), all others keep their
