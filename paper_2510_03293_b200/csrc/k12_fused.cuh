@@ -99,10 +99,12 @@ k12_route_select_tc(const RouteArgs A, int n_layers, const __grid_constant__ CUt
   if ((int)blockIdx.x < n_layers) {
     const int layer = A.layer0 + blockIdx.x;
     const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
-    // Measured: an SM that hosts a selection block starts no router block of this kernel (a
-    // resident block that never gives up its right to allocate tensor memory keeps the SM to
-    // itself).  That suits this kernel: the selection runs undisturbed at its own pace, and
-    // letting router blocks in (tcgen05.relinquish_alloc_permit here) made the launch slower.
+    // A resident block that never gives up its right to allocate tensor memory keeps router
+    // blocks of this kernel off its SM.  The selection role needs no tensor memory and, for the
+    // rule's own update order, is mostly waiting, so it gives the right up at once and router
+    // blocks share its SM.
+    if (threadIdx.x < 32)
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     k2_block<CMAX, false>(A, layer, dyn_smem, ready, kTcTileM);
     return;
   }

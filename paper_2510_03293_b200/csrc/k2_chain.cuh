@@ -42,10 +42,10 @@ __device__ __forceinline__ bool k2_wait_ready(const int* ready, int router_rows,
                                               int t_last, long long limit, bool block = true);
 
 __host__ __device__ inline int chain_cmax(int c) { return c <= 4 ? 4 : (c <= 8 ? 8 : (c <= 16 ? 16 : 32)); }
-// one slot: fb[E] int32 | fm[E] uint32 | ent[32][CMAX] u64 | ids[32][CMAX] u8 | out[32] u32 |
-// n, seq
+// one slot: fb[E] int32 | db[E] int32 | fm[E] uint32 | ent[32][CMAX] u64 | ids[32][CMAX] u8 |
+// out[32] u32 | n, seq, dl[32]
 __host__ __device__ inline size_t k2_chain_slot_bytes(int E, int cmax) {
-  return 2 * align256(sizeof(int32_t) * E) + (size_t)32 * cmax * 8 + (size_t)32 * cmax + 128 + 128;
+  return 3 * align256(sizeof(int32_t) * E) + (size_t)32 * cmax * 8 + (size_t)32 * cmax + 128 + 128;
 }
 // dcnt[E] | fcum[E] | counters | slots
 __host__ __device__ inline size_t k2_chain_smem_bytes(int E, int c) {
@@ -75,21 +75,54 @@ __device__ __forceinline__ int lds32(uint32_t a) {
 __device__ __forceinline__ void sts32(uint32_t a, int v) {
   asm volatile("st.shared.s32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
 }
-__device__ __forceinline__ int chain_ld_acquire(const int* p) {
+// hand-over words between the warps of the block
+__device__ __forceinline__ int lds_acquire(const int* p) {
   int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(chain_saddr(p)) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_release(int* p, int v) {
+  asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(chain_saddr(p)), "r"(v) : "memory");
+}
+// Loads that observe what other SMs have written (they do not hit a stale L1 line) without
+// ordering anything else: used to look at the router's flags and, once a flag has been seen
+// set, to fetch the records it covers (the router wrote them before releasing the flag).
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u16(const void* p) {
+  uint16_t v;
+  asm volatile("ld.relaxed.gpu.global.u16 %0, [%1];" : "=h"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u8(const void* p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u8 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint2 ld_relaxed_v2(const void* p) {
+  uint2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint4 ld_relaxed_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
 
 struct ChainSlot {
   int32_t* fb;                // [E] fixed assignments of this call made before the group
+  int32_t* db;                // [E] decisions of this call made before the group (by the chain)
   uint32_t* fm;               // [E] the group's masks of fixed tokens
   unsigned long long* ent;    // [32][CMAX] entries: load seen without decisions (all ones: no
                               //   candidate) | expert << 32 | cross-reference << 40 | token << 48
   uint8_t* ids;               // [32][CMAX] the group's ranked candidate ids (staging)
   uint32_t* out;              // [32] per entry: the chosen candidates (bit = lane)
-  int* n;                     // entries
-  int* seq;                   // group + 1 once the slot is ready for the chain
+  int* seq;                   // (group + 1) * 64 + entries once the slot is ready for the chain
   uint8_t* dl;                // [32] the group's decision tokens in order
 };
 
@@ -98,12 +131,12 @@ __device__ __forceinline__ ChainSlot chain_slot(unsigned char* slots, int slot, 
   unsigned char* p = slots + (size_t)slot * k2_chain_slot_bytes(E, CMAX);
   ChainSlot s;
   s.fb = reinterpret_cast<int32_t*>(p);              p += align256(sizeof(int32_t) * E);
+  s.db = reinterpret_cast<int32_t*>(p);              p += align256(sizeof(int32_t) * E);
   s.fm = reinterpret_cast<uint32_t*>(p);             p += align256(sizeof(int32_t) * E);
   s.ent = reinterpret_cast<unsigned long long*>(p);  p += (size_t)32 * CMAX * 8;
   s.ids = p;                                         p += (size_t)32 * CMAX;
   s.out = reinterpret_cast<uint32_t*>(p);            p += 128;
-  s.n = reinterpret_cast<int*>(p);
-  s.seq = s.n + 1;
+  s.seq = reinterpret_cast<int*>(p);
   s.dl = p + 32;
   return s;
 }
@@ -150,16 +183,26 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
     const uint32_t dcnt_a = chain_saddr(dcnt);
     for (int g = 0; g < n_groups; ++g) {
       const ChainSlot S = chain_slot<CMAX>(slots, g % kChainSlots, E);
-      while (ld_volatile_shared(S.seq) != g + 1) {
+      int word = lds_acquire(S.seq);
+      while ((word >> 6) != g + 1) {
         if (ld_volatile_shared(gave_up)) break;
         __nanosleep(20);
+        word = lds_acquire(S.seq);
       }
-      if (ld_volatile_shared(S.seq) != g + 1) break;   // the helpers gave up
-      __threadfence_block();
-      // base counts of the group: fixed assignments before it + decisions so far
-      int32_t* gb = g_base + (size_t)g * E;
-      for (int e = lane; e < E; e += 32) gb[e] = S.fb[e] + dcnt[e];
-      const int n = *S.n;
+      if ((word >> 6) != g + 1) break;   // the helpers gave up
+      const int n = word & 63;
+      // the decisions made before the group (the slot's helper adds the fixed assignments and
+      // writes the group's base counts to global memory; the chain itself stores nothing there)
+      {
+        const uint32_t db_a = chain_saddr(S.db) + 4u * lane;
+        int snap[MW];
+#pragma unroll
+        for (int q = 0; q < MW; ++q)
+          if (32 * q < E) snap[q] = lds32(dcnt_a + 4u * (lane + 32 * q));
+#pragma unroll
+        for (int q = 0; q < MW; ++q)
+          if (32 * q < E) sts32(db_a + 128u * q, snap[q]);
+      }
       if (n > 0) {
         // entry 0: its counters are exact (every earlier increment has landed).  Entries are
         // read two ahead and their counters one ahead (past the end: the last entry again).
@@ -204,7 +247,7 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
         }
       }
       __syncwarp();
-      if (lane == 0) { __threadfence_block(); st_volatile_shared(cons, g + 1); }
+      if (lane == 0) sts_release(cons, g + 1);
     }
   } else {
     // ---------------------------------------------------------------- the helpers
@@ -216,28 +259,39 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
       if (!ready || g >= n_groups) return ready ? 0 : 1;
       const int t0 = g * 32, rt_last = (min(T, t0 + 32) - 1) / router_rows;
       const int rt = min(t0 / router_rows + (router_rows < 32 ? (lane & 1) : 0), rt_last);
-      return chain_ld_acquire(ready + rt);
+      return (int)ld_relaxed_u32(ready + rt);
     };
     uint32_t mw[MW];      // the group's masks of experts lane, lane + 32, ...
     int cs = 0;           // c* of token lane
     uint4 idv = make_uint4(0, 0, 0, 0);   // its first 16 ranked ids (c <= 16)
     auto load_group = [&](int g) {
       const int t = g * 32 + lane;
-      cs = t < T ? (int)g_cs[t] : 0;
+      cs = t < T ? (int)ld_relaxed_u16(g_cs + t) : 0;
 #pragma unroll
       for (int q = 0; q < MW; ++q)
-        mw[q] = lane + 32 * q < E ? g_fm[(size_t)g * E + lane + 32 * q] : 0u;
+        mw[q] = lane + 32 * q < E ? ld_relaxed_u32(g_fm + (size_t)g * E + lane + 32 * q) : 0u;
       if (t < T && c <= 16) {
         const uint8_t* src = g_ids + (size_t)t * c;
-        if (c == 16) idv = *reinterpret_cast<const uint4*>(src);
-        else if (c == 8) { const uint2 v = *reinterpret_cast<const uint2*>(src); idv.x = v.x; idv.y = v.y; }
-        else if (c == 4) idv.x = *reinterpret_cast<const uint32_t*>(src);
+        if (c == 16) idv = ld_relaxed_v4(src);
+        else if (c == 8) { const uint2 v = ld_relaxed_v2(src); idv.x = v.x; idv.y = v.y; }
+        else if (c == 4) idv.x = ld_relaxed_u32(src);
         else {
           uint32_t wv[4] = {0, 0, 0, 0};
-          for (int r = 0; r < c; ++r) wv[r >> 2] |= (uint32_t)src[r] << (8 * (r & 3));
+          for (int r = 0; r < c; ++r) wv[r >> 2] |= ld_relaxed_u8(src + r) << (8 * (r & 3));
           idv = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
       }
+    };
+    // What the chain left in the slot for group g goes to global memory: the decision tokens'
+    // choices and the group's base counts (fixed assignments + decisions made before it).
+    auto flush = [&](int g, int n) {
+      if (lane < n) {
+        const int tok = (int)(S.ent[lane * CMAX] >> 48) & 31;
+        g_selmask[(size_t)g * 32 + tok] = S.out[lane];
+      }
+      int32_t* gb = g_base + (size_t)g * E;
+      for (int e = lane; e < E; e += 32) gb[e] = S.fb[e] + S.db[e];
+      __syncwarp();
     };
     bool ok = true;
     bool have = false;        // the records of this trip's group are already in registers
@@ -247,17 +301,14 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
       // the slot's previous group must have been consumed; its choices go to global memory
       if (g >= kChainSlots) {
         const long long start = clock64();
-        while (ld_volatile_shared(cons) < g - kChainSlots + 1) {
+        unsigned ns = 20;   // polls grow rarer: the chain shares this SM's shared-memory pipe
+        while (lds_acquire(cons) < g - kChainSlots + 1) {
           if (ld_volatile_shared(gave_up) || clock64() - start > A.wait_cycles) { ok = false; break; }
-          __nanosleep(500);   // (rare polls: the chain shares this SM's shared-memory pipe)
+          __nanosleep(ns);
+          ns = min(ns * 2u, 400u);
         }
         if (!ok) break;
-        __threadfence_block();
-        if (lane < n_prev) {
-          const int tok = (int)(S.ent[lane * CMAX] >> 48) & 31;
-          g_selmask[(size_t)(g - kChainSlots) * 32 + tok] = S.out[lane];
-        }
-        __syncwarp();
+        flush(g - kChainSlots, n_prev);
       }
       if (!have) {
         if (ready) {
@@ -283,7 +334,8 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
       } else {
         const int t = g * 32 + lane;
         if (t < T)
-          for (int r = 0; r < c; ++r) S.ids[lane * CMAX + r] = g_ids[(size_t)t * c + r];
+          for (int r = 0; r < c; ++r)
+            S.ids[lane * CMAX + r] = (uint8_t)ld_relaxed_u8(g_ids + (size_t)t * c + r);
       }
       const int my_cs = cs;
       // look ahead: if the next trip's group was seen published, request its records now (the
@@ -295,12 +347,11 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
       // the running count of fixed assignments: taken over from the group before, passed on
       {
         const long long start = clock64();
-        while (ld_volatile_shared(fdone) < g) {
+        while (lds_acquire(fdone) < g) {
           if (ld_volatile_shared(gave_up) || clock64() - start > A.wait_cycles) { ok = false; break; }
-          __nanosleep(100);
+          __nanosleep(20);
         }
         if (!ok) break;
-        __threadfence_block();
 #pragma unroll
         for (int q = 0; q < MW; ++q) {
           const int e = lane + 32 * q;
@@ -311,7 +362,7 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
           }
         }
         __syncwarp();
-        if (lane == 0) { __threadfence_block(); st_volatile_shared(fdone, g + 1); }
+        if (lane == 0) sts_release(fdone, g + 1);
       }
       // one entry per decision token, CMAX lanes each
       const unsigned dmask = __ballot_sync(0xffffffffu, my_cs > k);
@@ -353,28 +404,18 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
                               ((unsigned long long)x << 40) | ((unsigned long long)tokl << 48);
       }
       __syncwarp();
-      if (lane == 0) {
-        *S.n = n;
-        __threadfence_block();
-        st_volatile_shared(S.seq, g + 1);
-      }
+      if (lane == 0) sts_release(S.seq, (g + 1) * 64 + n);
       n_prev = n;
     }
     // the choices of the slot's last group
     if (ok && n_groups > hw) {
       const int g_last = hw + ((n_groups - 1 - hw) / kChainSlots) * kChainSlots;
       const long long start = clock64();
-      while (ld_volatile_shared(cons) < g_last + 1) {
+      while (lds_acquire(cons) < g_last + 1) {
         if (ld_volatile_shared(gave_up) || clock64() - start > A.wait_cycles) { ok = false; break; }
         __nanosleep(500);
       }
-      if (ok) {
-        __threadfence_block();
-        if (lane < n_prev) {
-          const int tok = (int)(S.ent[lane * CMAX] >> 48) & 31;
-          g_selmask[(size_t)g_last * 32 + tok] = S.out[lane];
-        }
-      }
+      if (ok) flush(g_last, n_prev);
     }
     if (!ok && lane == 0 && !ld_volatile_shared(gave_up)) fail();
   }
