@@ -36,15 +36,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 //   Z = eight interleaved running sums combined pairwise; s = e / Z;
 //   M_k = s_pi(0) + ... + s_pi(k-1) left to right; top-k branch iff M_k >= eps_high;
 //   otherwise c* = max(k, #{j < c : s_pi(j) >= t_fix * s_pi(0)}).
-// Writes the record (c*, ranked ids, ranked scores) for the load-aware scan and, for every
-// token, the top-k ids and weights (final for the top-k branch, overwritten otherwise).
+// Writes the record (c*, ranked ids, ranked scores) for the load-aware scan and the dispatch,
+// which derives every token's final ids and combine weights from it.
 // fm (shared memory, may be null): per-expert masks of the token's group; a token without a
 // load-dependent choice (top-k branch or c* == k) sets its bit for each of its k best.
 __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int E, int k, int c,
                                                float eps_high, float t_fix, int renorm,
                                                uint16_t* cstar, uint8_t* cand_ids,
-                                               float* cand_scores, int32_t* expert_ids,
-                                               float* weights, uint32_t* fm = nullptr,
+                                               float* cand_scores, uint32_t* fm = nullptr,
                                                uint32_t bit = 0) {
   float xmax = x[0];
   for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, x[i]);
@@ -79,15 +78,11 @@ __device__ __forceinline__ void token_epilogue(const float* __restrict__ x, int 
     if (s >= thr) ++mprime;
     cand_ids[r] = (uint8_t)bi;
     cand_scores[r] = s;
-    if (r < k) { expert_ids[r] = bi; weights[r] = s; }
     prev_x = bx;
     prev_i = bi;
   }
   const bool top_k_branch = (Mk >= eps_high);
   *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
-  if (top_k_branch && renorm) {
-    for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
-  }
   if (fm && (top_k_branch || mprime <= k))
     for (int j = 0; j < k; ++j) atomicOr(&fm[cand_ids[j]], bit);   // (reads its own stores)
 }
@@ -122,8 +117,7 @@ static __device__ __noinline__ void token_epilogue_random(const float* row, int 
                                                    float eps_high, float t_fix, int renorm,
                                                    unsigned long long seed, int layer, long long t,
                                                    uint16_t* cstar, uint8_t* cand_ids,
-                                                   float* cand_scores, int32_t* expert_ids,
-                                                   float* weights, uint32_t* fm = nullptr,
+                                                   float* cand_scores, uint32_t* fm = nullptr,
                                                    uint32_t bit = 0) {
   float xmax = row[0];
   for (int i = 1; i < E; ++i) xmax = fmaxf(xmax, row[i]);
@@ -161,8 +155,6 @@ static __device__ __noinline__ void token_epilogue_random(const float* row, int 
     if (r < k) {
       const float s = __fdiv_rn(exp32(__fsub_rn(bx, xmax)), Z);
       Mk = r == 0 ? s : __fadd_rn(Mk, s);
-      expert_ids[r] = bi;
-      weights[r] = s;
       cand_ids[r] = (uint8_t)bi;   // the top-k branch's record: the selection and the dispatch
       cand_scores[r] = s;          // read the k best from here (overwritten by a sample)
       if (r == k - 1 && !(Mk >= eps_high)) need = m;   // expanded: rank the whole pool
@@ -172,8 +164,6 @@ static __device__ __noinline__ void token_epilogue_random(const float* row, int 
   }
   if (Mk >= eps_high) {
     *cstar = 0;
-    if (renorm)
-      for (int j = 0; j < k; ++j) weights[j] = __fdiv_rn(weights[j], Mk);
     if (fm)
       for (int j = 0; j < k; ++j) atomicOr(&fm[cand_ids[j]], bit);
     return;
@@ -260,7 +250,6 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
                                                       int c, float eps_high, float t_fix,
                                                       int renorm, uint16_t* cstar,
                                                       uint8_t* cand_ids, float* cand_scores,
-                                                      int32_t* expert_ids, float* weights,
                                                       uint32_t* fm = nullptr, uint32_t bit = 0) {
   constexpr uint32_t IDX = N - 1;
   constexpr int SH = N == 64 ? 6 : 7;
@@ -328,8 +317,7 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
     }
   }
   if (!exact) {
-    token_epilogue(row, E, k, c, eps_high, t_fix, renorm, cstar, cand_ids, cand_scores, expert_ids,
-                   weights, fm, bit);
+    token_epilogue(row, E, k, c, eps_high, t_fix, renorm, cstar, cand_ids, cand_scores, fm, bit);
     return;
   }
   float Mk = 0.0f, thr = 0.0f;
@@ -354,17 +342,12 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
     for (int r = 0; r < CL; ++r)
       if (r < k) atomicOr(&fm[IDX - (R[r] & IDX)], bit);
   }
-  float wv[CL];   // combine weights of the k best
-#pragma unroll
-  for (int r = 0; r < CL; ++r) wv[r] = (top_k_branch && renorm) ? __fdiv_rn(sv[r], Mk) : sv[r];
-  // Records out.  With c = 8 and an even k (the shapes this epilogue mostly sees) a token's
-  // record is written with 8- and 16-byte stores: the stores of a warp go to 32 different
-  // sectors each, so their number is what costs.
+  // Records out (the final ids and weights of every token are written by the dispatch).  With
+  // c = 8 a token's record is written with 8- and 16-byte stores: the stores of a warp go to 32
+  // different sectors each, so their number is what costs.
   if constexpr (CL == 8) {
-    // (the scratch records are 8 and 32 bytes per token in a 256-byte aligned workspace; the
-    // caller's id and weight arrays only promise 4-byte alignment, hence the test)
-    if (c == 8 && (k & 1) == 0 &&
-        ((reinterpret_cast<uintptr_t>(expert_ids) | reinterpret_cast<uintptr_t>(weights)) & 7) == 0) {
+    // (the scratch records are 8 and 32 bytes per token in a 256-byte aligned workspace)
+    if (c == 8) {
       uint32_t lo = 0, hi = 0;
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
@@ -374,14 +357,6 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
       *reinterpret_cast<uint2*>(cand_ids) = make_uint2(lo, hi);
       *reinterpret_cast<float4*>(cand_scores) = make_float4(sv[0], sv[1], sv[2], sv[3]);
       *reinterpret_cast<float4*>(cand_scores + 4) = make_float4(sv[4], sv[5], sv[6], sv[7]);
-#pragma unroll
-      for (int r = 0; r < CL; r += 2) {
-        if (r < k) {
-          *reinterpret_cast<int2*>(expert_ids + r) =
-              make_int2((int)(IDX - (R[r] & IDX)), (int)(IDX - (R[r + 1] & IDX)));
-          *reinterpret_cast<float2*>(weights + r) = make_float2(wv[r], wv[r + 1]);
-        }
-      }
       return;
     }
   }
@@ -391,7 +366,6 @@ __device__ __forceinline__ void token_epilogue_sorted(const float* __restrict__ 
       const int bi = (int)(IDX - (R[r] & IDX));
       cand_ids[r] = (uint8_t)bi;
       cand_scores[r] = sv[r];
-      if (r < k) { expert_ids[r] = bi; weights[r] = wv[r]; }
     }
   }
 }
@@ -409,7 +383,6 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
                                                       float eps_high, float t_fix, int renorm,
                                                       bool write, uint16_t* cstar,
                                                       uint8_t* cand_ids, float* cand_scores,
-                                                      int32_t* expert_ids, float* weights,
                                                       uint32_t* fm = nullptr, uint32_t bit = 0) {
   constexpr int EPL = N / 8;
   const float ninf = __int_as_float(0xff800000);
@@ -461,7 +434,6 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
       if (write && j == 0) {
         cand_ids[r] = (uint8_t)bi;
         cand_scores[r] = sr;
-        if (r < k) { expert_ids[r] = bi; weights[r] = sr; }
       }
       prev_x = bx;
       prev_i = bi;
@@ -469,8 +441,6 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
     if (!write || j != 0) return;
     const bool top_k_branch = (Mk >= eps_high);
     *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
-    if (top_k_branch && renorm)
-      for (int q = 0; q < k; ++q) weights[q] = __fdiv_rn(weights[q], Mk);
     if (fm && (top_k_branch || mprime <= k))
       for (int q = 0; q < k; ++q) atomicOr(&fm[cand_ids[q]], bit);
     return;
@@ -539,10 +509,6 @@ __device__ __forceinline__ void token_epilogue_lanes8(const float* row, int j, i
     if (r < c) {
       cand_ids[r] = (uint8_t)ki[q];
       cand_scores[r] = sc[q];
-      if (r < k) {
-        expert_ids[r] = ki[q];
-        weights[r] = (top_k_branch && renorm) ? __fdiv_rn(sc[q], Mk) : sc[q];
-      }
     }
   }
   if (j == 0) *cstar = top_k_branch ? (uint16_t)0 : (uint16_t)max(k, mprime);
@@ -708,17 +674,16 @@ __device__ __forceinline__ void group_epilogue(const RouteArgs& A, int layer, lo
   if (t < A.T) {
     unsigned char* ws = A.ws + (size_t)(A.layer0 + layer) * A.ws_ls;
     const int k = A.k, c = A.c;
-    const size_t lt = (size_t)(A.layer0 + layer) * A.T + t;
     uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
     uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
     float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
     if (A.trim_random)
       token_epilogue_random(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer],
-                            A.renorm, A.seed, A.layer0 + layer, t, cs_p, ids_p, sc_p,
-                            A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
+                            A.renorm, A.seed, A.layer0 + layer, t, cs_p, ids_p, sc_p, fm,
+                            1u << lane);
     else
       token_epilogue(rows + lane * lds, A.E, k, c, A.eps_high[layer], A.t_fix[layer], A.renorm,
-                     cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
+                     cs_p, ids_p, sc_p, fm, 1u << lane);
   }
   if (masks) publish_group_masks(A, A.layer0 + layer, tok0, fm, lane);
 }
@@ -852,13 +817,12 @@ __device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int laye
     if (tid < 16 && t < T) {
       unsigned char* ws = A.ws + (size_t)abs_layer * A.ws_ls;
       const int k = A.k, c = A.c;
-      const size_t lt = (size_t)abs_layer * T + t;
       token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer],
                             A.renorm, A.seed, abs_layer, t,
                             reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
                             ws + A.lay.cand_ids + (size_t)t * c,
                             reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
-                            A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << tid);
+                            fm, 1u << tid);
     }
   } else if (warp < 4) {
     const int r = warp * 4 + (lane >> 3);
@@ -867,13 +831,12 @@ __device__ __forceinline__ void router_splitk_block(const RouteArgs& A, int laye
     const long long tc = write ? t : 0;
     unsigned char* ws = A.ws + (size_t)abs_layer * A.ws_ls;
     const int k = A.k, c = A.c;
-    const size_t lt = (size_t)abs_layer * T + tc;
     token_epilogue_lanes8<EP>(tile + (size_t)r * LDS, lane & 7, E, k, c, A.eps_high[layer],
                               A.t_fix[layer], A.renorm, write,
                               reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + tc,
                               ws + A.lay.cand_ids + (size_t)tc * c,
                               reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)tc * c,
-                              A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << r);
+                              fm, 1u << r);
   }
   if (fm) {
     __syncthreads();

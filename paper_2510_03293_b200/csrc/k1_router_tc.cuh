@@ -285,22 +285,20 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
       const long long t = tok0 + tid;
       uint32_t* fm = s_fm + warp * N;   // warps 0..3 each score one group of 32 tokens
       if (tid < kTcTileM && t < T) {
-        const size_t lt = (size_t)abs_layer * T + t;
         uint16_t* cs_p = reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t;
         uint8_t* ids_p = ws + A.lay.cand_ids + (size_t)t * c;
         float* sc_p = reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c;
         if (A.trim_random)
           token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
                                 A.t_fix[layer], A.renorm, A.seed, abs_layer, t, cs_p, ids_p, sc_p,
-                                A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
+                                fm, 1u << lane);
         else if (c <= CL)
           token_epilogue_sorted<N, CL>(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
-                                       A.t_fix[layer], A.renorm, cs_p, ids_p, sc_p,
-                                       A.expert_ids + lt * k, A.weights + lt * k, fm, 1u << lane);
+                                       A.t_fix[layer], A.renorm, cs_p, ids_p, sc_p, fm,
+                                       1u << lane);
         else
           token_epilogue(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer], A.t_fix[layer],
-                         A.renorm, cs_p, ids_p, sc_p, A.expert_ids + lt * k, A.weights + lt * k,
-                         fm, 1u << lane);
+                         A.renorm, cs_p, ids_p, sc_p, fm, 1u << lane);
       }
       if (warp < 4 && tok0 + warp * 32 < T)
         publish_group_masks(A, abs_layer, tok0 + warp * 32, fm, lane);
@@ -341,13 +339,11 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
       if (A.trim_random) {   // one thread per token of this pass
         const long long t = tok0 + tid;
         if (tid < ROWS && t < T) {
-          const size_t lt = (size_t)abs_layer * T + t;
           token_epilogue_random(tile + (size_t)tid * LDS, E, k, c, A.eps_high[layer],
                                 A.t_fix[layer], A.renorm, A.seed, abs_layer, t,
                                 reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + t,
                                 ws + A.lay.cand_ids + (size_t)t * c,
                                 reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)t * c,
-                                A.expert_ids + lt * k, A.weights + lt * k,
                                 s_fm + ((row0 + tid) >> 5) * N, 1u << (tid & 31));
         }
       }
@@ -359,13 +355,11 @@ __device__ __forceinline__ bool router_tc_block(const RouteArgs& A, const CUtens
         const long long t = tok0 + r;
         const bool write = t < T;
         const long long tc = write ? t : 0;   // keeps the pointers of idle groups in bounds
-        const size_t lt = (size_t)abs_layer * T + tc;
         token_epilogue_lanes8<N>(tile + (size_t)r * LDS, j, E, k, c, A.eps_high[layer],
                                  A.t_fix[layer], A.renorm, write,
                                  reinterpret_cast<uint16_t*>(ws + A.lay.cstar) + tc,
                                  ws + A.lay.cand_ids + (size_t)tc * c,
                                  reinterpret_cast<float*>(ws + A.lay.cand_scores) + (size_t)tc * c,
-                                 A.expert_ids + lt * k, A.weights + lt * k,
                                  s_fm + ((row0 + r) >> 5) * N, 1u << (r & 31));
       }
       __syncthreads();   // the tile is reused by the next pass

@@ -9,7 +9,7 @@
 // which is also the load increment that token saw.  The warp first builds, per expert, the bit
 // mask of its tokens sent there (the second term is then a population count), then every lane
 // finishes its own token:
-//   top-k branch (c* = 0): slots in score order; ids and weights were written by the router.
+//   top-k branch (c* = 0): slots in score order.
 //   c* > k: slots as the load-aware scan listed them (ascending load, then score rank); where
 //           the scan left the choice as a bit mask over score ranks (the layer's mode word is
 //           set), the slot order is rebuilt like that of c* == k.
@@ -57,53 +57,84 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
   const bool as_masks =
       reinterpret_cast<const int*>(ws + A.lay.ready)[mode_word_index(T)] != 0;
 
-  for (int e = lane; e < E; e += 32) { base[e] = gb[e]; mask[e] = 0; }
+  // Everything a token can need is requested at once, whatever its branch turns out to be, so
+  // that the group costs one round trip to memory: c*, the first KR ranked ids and scores, the
+  // chosen ranks of a decision token, and per expert the group's base count and (E > 32) the
+  // router's mask of the group's tokens without a decision.
+  const float* sc = reinterpret_cast<const float*>(ws + A.lay.cand_scores) + (size_t)t * c;
+  const bool have_fm = E > 32;
+  const uint32_t* fmg = reinterpret_cast<const uint32_t*>(ws + A.lay.fmask) + (size_t)g * E;
+  int idr[KR];
+  float scr[KR];
+  uint32_t chosen = 0;
+#pragma unroll
+  for (int j = 0; j < KR; ++j) { idr[j] = 0; scr[j] = 0.0f; }
+  if (valid) {
+    if (c == 8 && KR <= 8) {
+      const uint2 v = *reinterpret_cast<const uint2*>(cand);
+#pragma unroll
+      for (int j = 0; j < KR; ++j) idr[j] = (int)(((j < 4 ? v.x : v.y) >> (8 * (j & 3))) & 255u);
+    } else if (c == 4 && KR <= 4) {
+      const uint32_t v = *reinterpret_cast<const uint32_t*>(cand);
+#pragma unroll
+      for (int j = 0; j < KR; ++j) idr[j] = (int)((v >> (8 * j)) & 255u);
+    } else {
+#pragma unroll
+      for (int j = 0; j < KR; ++j)
+        if (j < c) idr[j] = cand[j];
+    }
+    if (c % 4 == 0 && KR >= 4) {   // 16-byte aligned records: one or two full-width loads
+      const float4 lo = *reinterpret_cast<const float4*>(sc);
+      scr[0] = lo.x; scr[1] = lo.y; scr[2] = lo.z; scr[3] = lo.w;
+      if constexpr (KR == 8) {
+        if (c >= 8) {
+          const float4 hi = *reinterpret_cast<const float4*>(sc + 4);
+          scr[4] = hi.x; scr[5] = hi.y; scr[6] = hi.z; scr[7] = hi.w;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < KR; ++j)
+        if (j < c) scr[j] = sc[j];
+    }
+    if (have_fm) chosen = reinterpret_cast<const uint32_t*>(ws + A.lay.sel_mask)[t];   // (used if as_masks)
+  }
+  for (int e = lane; e < E; e += 32) { base[e] = gb[e]; mask[e] = have_fm ? fmg[e] : 0u; }
   __syncwarp();
   int ex[KR], rk[KR];   // expert and candidate rank of slot j as the selection listed them
+  float sr[KR];         // and its score
 #pragma unroll
-  for (int j = 0; j < KR; ++j) { ex[j] = 0; rk[j] = j; }
-  if (valid) {
-    uint32_t chosen = (cs > k && as_masks)
-                          ? reinterpret_cast<const uint32_t*>(ws + A.lay.sel_mask)[t] : 0u;
+  for (int j = 0; j < KR; ++j) { ex[j] = idr[j]; rk[j] = j; sr[j] = scr[j]; }
+  if (valid && cs > k) {   // a decision token: its ranks, experts and scores (few tokens)
 #pragma unroll
     for (int j = 0; j < KR; ++j)
       if (j < k) {
-        if (cs > k) {
-          if (as_masks) { rk[j] = __ffs(chosen) - 1; chosen &= chosen - 1; }   // ascending rank
-          else rk[j] = sel[j];
-        }
+        if (as_masks) { rk[j] = __ffs(chosen) - 1; chosen &= chosen - 1; }   // ascending rank
+        else rk[j] = sel[j];
         ex[j] = cand[rk[j]];
-        atomicOr(&mask[ex[j]], 1u << lane);
+        sr[j] = sc[rk[j]];
       }
   }
+  if (valid && (!have_fm || cs > k)) {
+#pragma unroll
+    for (int j = 0; j < KR; ++j)
+      if (j < k) atomicOr(&mask[ex[j]], 1u << lane);
+  }
   __syncwarp();
-  if (!valid) return;
   const unsigned below = (1u << lane) - 1;
   int pos[KR];
 #pragma unroll
-  for (int j = 0; j < KR; ++j) pos[j] = j < k ? base[ex[j]] + __popc(mask[ex[j]] & below) : 0;
+  for (int j = 0; j < KR; ++j)
+    pos[j] = (valid && j < k) ? base[ex[j]] + __popc(mask[ex[j]] & below) : 0;
 
-  const float* sc = reinterpret_cast<const float*>(ws + A.lay.cand_scores) + (size_t)t * c;
   int32_t* perm = A.perm + (size_t)layer * T * k;
-  int32_t* ids = A.expert_ids + ((size_t)layer * T + t) * k;
-  float* w = A.weights + ((size_t)layer * T + t) * k;
   const int32_t pair0 = (int32_t)(t * k);
-
-  if (cs == 0) {   // top-k branch: ids and weights were written by the router
-#pragma unroll
-    for (int j = 0; j < KR; ++j)
-      if (j < k) perm[off_s[ex[j]] + pos[j]] = pair0 + j;
-    return;
-  }
   float v[KR];     // weights in slot order
   int slot[KR];
 #pragma unroll
-  for (int j = 0; j < KR; ++j) { v[j] = 0.0f; slot[j] = j; }
-  if (cs > k && !as_masks) {
-#pragma unroll
-    for (int j = 0; j < KR; ++j)
-      if (j < k) v[j] = sc[rk[j]];
-  } else {
+  for (int j = 0; j < KR; ++j) { v[j] = sr[j]; slot[j] = j; }
+  // top-k branch (c* = 0): score order, as ranked.  c* > k listed by the selection: as listed.
+  if (valid && cs != 0 && !(cs > k && !as_masks)) {
     // the set is known, in ascending score rank (c* == k: the k best): slots by (load seen,
     // score rank); the load seen by the expert of rank j is L_in[e] + position
     // (relaxed variant: + the assignments made before the token's chunk instead)
@@ -112,12 +143,9 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
       gb0 = reinterpret_cast<const int32_t*>(ws + A.lay.grp_base) +
             (size_t)(A.G == 0 ? 0 : ((t / A.G) * A.G) / 32) * E;
     int32_t seen[KR];
-    float sj[KR];
 #pragma unroll
-    for (int j = 0; j < KR; ++j) {
+    for (int j = 0; j < KR; ++j)
       seen[j] = j < k ? lin_s[ex[j]] + (gb0 ? gb0[ex[j]] : pos[j]) : 0;
-      sj[j] = j < k ? sc[rk[j]] : 0.0f;
-    }
 #pragma unroll
     for (int j = 0; j < KR; ++j) {
       int sl = 0;
@@ -130,20 +158,32 @@ __device__ __forceinline__ void k3_group_regs(const RouteArgs& A, int layer, int
     for (int s2 = 0; s2 < KR; ++s2) {
 #pragma unroll
       for (int j = 0; j < KR; ++j)
-        if (j < k && slot[j] == s2) v[s2] = sj[j];
+        if (j < k && slot[j] == s2) v[s2] = sr[j];
     }
   }
   float sum = v[0];
 #pragma unroll
   for (int j = 1; j < KR; ++j)
     if (j < k) sum = __fadd_rn(sum, v[j]);
+  // ids and weights of the group's tokens are one contiguous block each: staged in shared
+  // memory in slot order and written with full-width stores (the router's own copy of the
+  // top-k branch's ids and weights is the same bits: its M_k is this left-to-right sum)
+  int32_t* ids_s = base + 2 * E;
+  float* w_s = reinterpret_cast<float*>(ids_s + 32 * k);
+  if (valid) {
 #pragma unroll
-  for (int j = 0; j < KR; ++j)
-    if (j < k) {
-      ids[slot[j]] = ex[j];
-      perm[off_s[ex[j]] + pos[j]] = pair0 + slot[j];
-      w[j] = A.renorm ? __fdiv_rn(v[j], sum) : v[j];
-    }
+    for (int j = 0; j < KR; ++j)
+      if (j < k) {
+        ids_s[lane * k + slot[j]] = ex[j];
+        w_s[lane * k + j] = A.renorm ? __fdiv_rn(v[j], sum) : v[j];
+        perm[off_s[ex[j]] + pos[j]] = pair0 + slot[j];
+      }
+  }
+  __syncwarp();
+  const int n_out = (int)min(32LL, (long long)T - (long long)g * 32) * k;
+  int32_t* ids = A.expert_ids + ((size_t)layer * T + (size_t)g * 32) * k;
+  float* w = A.weights + ((size_t)layer * T + (size_t)g * 32) * k;
+  for (int i = lane; i < n_out; i += 32) { ids[i] = ids_s[i]; w[i] = w_s[i]; }
 }
 
 // Group g (32 tokens) of absolute layer `layer`, by one warp.  lin_s / off_s: the layer's loads
@@ -210,12 +250,16 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
   const int32_t* mypos = pos + lane * k;
   const uint8_t* mype = pe + lane * k;
 
-  if (cs == 0) {
-    for (int j = 0; j < k; ++j) perm[off[mype[j]] + mypos[j]] = pair0 + j;
-    return;
-  }
   float sum = 0.0f;
-  if (cs > k && !as_masks) {
+  if (cs == 0) {   // top-k branch: score order, M_k = the left-to-right sum of the k best
+    for (int j = 0; j < k; ++j) {
+      const float v = sc[j];
+      ids[j] = mype[j];
+      w[j] = v;
+      sum = j == 0 ? v : __fadd_rn(sum, v);
+      perm[off[mype[j]] + mypos[j]] = pair0 + j;
+    }
+  } else if (cs > k && !as_masks) {
     for (int j = 0; j < k; ++j) {
       const int e = mype[j];
       ids[j] = e;
