@@ -65,9 +65,9 @@ DECODE_NODES_PER_CALL = 2   # a memset of the router's flags and one kernel
 
 def launches_per_step(w, L) -> int:
     """Kernels the library enqueues per step, per group of at most 64 layers: the fused
-    router + selection kernel and the dispatch kernel (calls of at most 256 tokens have their
+    router + selection kernel and the dispatch kernel (calls of at most 512 tokens have their
     dispatch done inside the first kernel)."""
-    return (1 if w.T <= 256 else 2) * ((L + 63) // 64)
+    return (1 if w.T <= 512 else 2) * ((L + 63) // 64)
 
 
 def kernel_sources_digest() -> str:

@@ -352,14 +352,20 @@ __device__ __forceinline__ void k2_chain_layer(const RouteArgs& A, int layer, un
           __nanosleep(20);
         }
         if (!ok) break;
+        {
+          // all loads first, then the stores (explicit shared-memory accesses: nothing here
+          // waits for a store to land before the next load)
+          const uint32_t fc_a = chain_saddr(fcum) + 4u * lane, fb_a = chain_saddr(S.fb) + 4u * lane;
+          int f[MW];
 #pragma unroll
-        for (int q = 0; q < MW; ++q) {
-          const int e = lane + 32 * q;
-          if (e < E) {
-            const int f = fcum[e];
-            S.fb[e] = f;
-            fcum[e] = f + cnt[q];
-          }
+          for (int q = 0; q < MW; ++q)
+            if (32 * q < E) f[q] = lds32(fc_a + 128u * q);
+#pragma unroll
+          for (int q = 0; q < MW; ++q)
+            if (32 * q < E) {
+              sts32(fc_a + 128u * q, f[q] + cnt[q]);
+              sts32(fb_a + 128u * q, f[q]);
+            }
         }
         __syncwarp();
         if (lane == 0) sts_release(fdone, g + 1);

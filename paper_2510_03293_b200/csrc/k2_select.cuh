@@ -68,7 +68,7 @@ __host__ __device__ inline size_t k2_smem_bytes(int E, int c, int k) {
 
 // Calls of at most this many 32-token groups have their dispatch done by the selection block
 // itself (one launch less); its scratch lies behind L, Lin and Lvis in the selection's memory.
-constexpr int kFusedDispatchGroups = 8;
+constexpr int kFusedDispatchGroups = 16;
 __host__ __device__ inline size_t k2_fused_dispatch_bytes(int E, int k) {
   return 3 * align256(sizeof(int32_t) * E) + (size_t)kK2Warps * k3_warp_smem_bytes(E, k);
 }
