@@ -897,6 +897,8 @@ def main():
                     help="one workload only (tiny, mixtral, deepseek, decode, stress); default: "
                          "mixtral as the line's value with the other four under 'workloads'")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count")
+    ap.add_argument("--tokens", type=int, default=None,
+                    help="override the tokens per layer (small cases for profiling)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-layers", type=int, default=8)
@@ -942,6 +944,8 @@ def main():
             over["t_fix"] = args.t_fix
         if args.c is not None:
             over["c"] = args.c
+        if args.tokens is not None:
+            over["T"] = args.tokens
         return dataclasses_replace(w, **over) if over else w
 
     headline = args.workload or "mixtral"
@@ -951,7 +955,7 @@ def main():
     ctx = Context()
     run = lambda w, full: (run_decode if w.persistent_loads else run_layers)(args, w, ctx, full)
     result = run(workload(headline), True)
-    if args.workload is None and ctx.world == 1 and args.layers is None:
+    if args.workload is None and ctx.world == 1 and args.layers is None and args.tokens is None:
         subs = {}
         for name in SUB_WORKLOADS:
             r = run(workload(name), False)

@@ -303,7 +303,7 @@ __device__ __forceinline__ void k3_group(const RouteArgs& A, int layer, int g,
 
 // (defined in one translation unit only: the one that launches it)
 #ifdef LASER_DEFINE_K3_KERNEL
-__global__ void k3_dispatch(const RouteArgs A) {
+__global__ void __launch_bounds__(256, 5) k3_dispatch(const RouteArgs A) {
   extern __shared__ __align__(16) unsigned char k3_smem[];
   const int layer = A.layer0 + blockIdx.y;
   const int warp = threadIdx.x >> 5;
