@@ -287,7 +287,7 @@ enum { LASER_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 };
  *   - The call itself allocates and frees nothing, on the host side of CUDA or the device.
  *   - Parameters whose laser_workspace_bytes() is larger than LASER_STATIC_SCRATCH_BYTES are
  *     refused with LASER_ERR_STATIC_SCRATCH and nothing is launched.  One layer of 16384
- *     tokens with k = 6, c = 8 needs about 2.3 MiB.
+ *     tokens with k = 6, c = 8 needs about 1.1 MiB.
  *   - The device that owns cuda_stream must be the current device.
  *   - The first call on each device looks up the array's device address (a runtime query,
  *     once per device, cached under a lock).  Make that first call outside any stream

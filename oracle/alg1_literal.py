@@ -2,9 +2,10 @@
 
 TEST INFRASTRUCTURE, not a product path.  Three independent pieces:
 
-* ``alg1_token``   -- Algorithm 1 of the paper taken literally: a candidate *set* built by
-  thresholding all n scores, united with the top-k, trimmed to the c* highest-scoring, then
-  a stable sort by load with score as tie-break.
+* ``alg1_token``   -- the routing rule of Algorithm 1 stated as set definitions over all n
+  experts (pool membership, candidates as the pool members with fewer than c pool members
+  ahead of them, the choice as the candidates with fewer than k smaller (load, rank) keys),
+  evaluated by counting; nothing is sorted or trimmed step by step.
 * ``brute_force_token`` -- the selection step by exhaustive search: among all k-subsets of
   the candidate set, the one whose sorted (load, score-rank) key vector is smallest.
 * ``imbalance`` / ``max_violation`` -- the imbalance factor of Motivation and MV of
@@ -26,29 +27,35 @@ def score_order(s, x=None):
 
 
 def alg1_token(s, L, k, c, eps_high, t_fix, x=None):
-    """Algorithm 1 (TOP trimming) for one token.  s: fp32 scores, L: integer loads.
+    """The routing rule for one token (Algorithm 1 with TOP trimming is the source of the rule),
+    written as definitions over all n experts rather than as a procedure.  s: fp32 scores,
+    L: integer loads.
 
-    Returns (A as a list in the order the sorted candidate list yields, expanded flag,
-    c*).  All comparisons on scores are made in fp32, as the scores are given.
+      peaked      the k best scores add up (fp32, best first) to at least eps_high
+      in the pool an expert is one of the k best, or its score reaches t_fix times the best score
+      candidate   a pool member with fewer than c pool members ranked ahead of it by score
+      chosen      a candidate with fewer than k candidates whose (load, score rank) is smaller
+
+    Returns (the chosen experts by ascending (load, score rank) -- for a peaked token the k
+    best by score --, expanded flag, number of candidates).  All comparisons on scores are
+    made in fp32, as the scores are given.
     """
     s = np.asarray(s, np.float32)
     n = len(s)
-    order = score_order(s, x)
-    Mk = np.float32(s[order[0]])
-    for j in range(1, k):
-        Mk = np.float32(Mk + s[order[j]])
-    if Mk >= np.float32(eps_high):
-        return list(order[:k]), False, 0
-    t = np.float32(np.float32(t_fix) * s[order[0]])
-    pool = {i for i in range(n) if s[i] >= t} | set(order[:k])
-    m = len(pool)
-    c_star = min(c, m)
-    by_score = [i for i in order if i in pool]
-    cand = by_score[:c_star]
-    # stable sort by load; cand is already in descending score order, so stability
-    # realises "ties broken by score, descending".
-    cand_sorted = sorted(cand, key=lambda i: int(L[i]))
-    return cand_sorted[:k], True, c_star
+    rank = {i: r for r, i in enumerate(score_order(s, x))}
+    best = [i for i in range(n) if rank[i] < k]
+    best.sort(key=rank.get)
+    mass = np.float32(s[best[0]])
+    for i in best[1:]:
+        mass = np.float32(mass + s[i])
+    if mass >= np.float32(eps_high):
+        return best, False, 0
+    floor = np.float32(np.float32(t_fix) * s[best[0]])
+    pool = [i for i in range(n) if rank[i] < k or s[i] >= floor]
+    cand = [i for i in pool if sum(rank[j] < rank[i] for j in pool) < c]
+    key = lambda i: (int(L[i]), rank[i])
+    chosen = [i for i in cand if sum(key(j) < key(i) for j in cand) < k]
+    return sorted(chosen, key=key), True, len(cand)
 
 
 def alg1_sequence(S, loads, k, c, eps_high, t_fix, X=None):
