@@ -13,14 +13,20 @@
 extern "C" {
 #endif
 
-enum { LASER_TEST_ROUTER_AUTO = 0, LASER_TEST_ROUTER_TILE = 1, LASER_TEST_ROUTER_SPLITK = 2 };
+enum {
+  LASER_TEST_ROUTER_AUTO = 0,
+  LASER_TEST_ROUTER_TILE = 1,          /* the 128-token-tile routers */
+  LASER_TEST_ROUTER_SPLITK = 2,        /* the 16-token split-K router */
+  LASER_TEST_ROUTER_TILE_ONESHOT = 3   /* as TILE, but 32 < E <= 64 takes the one-tile-per-block
+                                          form of the tensor-memory router, not the persistent one */
+};
 
 /*
  * Overrides the choice between the 128-token-tile routers and the 16-token split-K router,
  * which is otherwise made from the number of tokens, so that small test shapes can run through
  * both.  It changes speed, never decisions (logits may differ in the last bits, as between any
  * two summation orders).  Returns the previous mode, or -1 (and changes nothing) for a mode
- * that is none of the three above.
+ * that is none of those above.
  */
 int laser_test_set_router(int mode);
 

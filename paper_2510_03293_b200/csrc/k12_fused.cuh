@@ -9,6 +9,7 @@
 #include "k1_router.cuh"
 #include "k2_select.cuh"
 #include "k1_router_tc.cuh"
+#include "k1_router_tcp.cuh"
 
 namespace laser {
 
@@ -121,6 +122,28 @@ k12_route_select_tc(const RouteArgs A, int n_layers, const __grid_constant__ CUt
     __threadfence();
     st_release(ready + rt, done ? 1 : -1);
   }
+}
+
+// The persistent form of the tensor-memory router (E <= 128): the first n_layers blocks select,
+// every other block walks the tiles b, b + P, ... of all layers (tile id = tile index * n_layers
+// + layer).
+template <int N, int CMAX>
+__global__ void __launch_bounds__(kK2Threads, 2)
+k12_route_select_tcp(const RouteArgs A, int n_layers, int n_tiles,
+                     const __grid_constant__ CUtensorMap map_h,
+                     const __grid_constant__ CUtensorMap map_w) {
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
+  if ((int)blockIdx.x < n_layers) {
+    const int layer = A.layer0 + blockIdx.x;
+    const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
+    if (threadIdx.x < 32)   // the selection needs no tensor memory: router blocks share its SM
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    k2_block<CMAX, false>(A, layer, dyn_smem, ready, kTcTileM);
+    return;
+  }
+  router_tcp_block<N, (CMAX < 8 ? 8 : CMAX)>(A, &map_h, &map_w, n_layers,
+                                             (int)blockIdx.x - n_layers,
+                                             (int)gridDim.x - n_layers, n_tiles, dyn_smem);
 }
 
 }  // namespace laser

@@ -54,6 +54,32 @@ cudaError_t launch_k12_tc(const RouteArgs& a, int n_layers, const CUtensorMap& m
   return cudaGetLastError();
 }
 
+// Persistent form (N <= 128): router_blocks blocks walk all tiles of the launch.
+template <int N, int CMAX>
+cudaError_t launch_k12_tcp(const RouteArgs& a, int n_layers, int router_blocks,
+                           const CUtensorMap& mh, const CUtensorMap& mw, cudaStream_t s) {
+  size_t smem = tcp_smem_bytes<N>();
+  const size_t smem2 = selection_smem(a);
+  if (smem2 > smem) smem = smem2;
+  cudaError_t e = cudaFuncSetAttribute(k12_route_select_tcp<N, CMAX>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const int n_tiles = n_layers * ((a.T + kTcTileM - 1) / kTcTileM);
+  if (router_blocks > n_tiles) router_blocks = n_tiles;
+  k12_route_select_tcp<N, CMAX>
+      <<<n_layers + router_blocks, kK2Threads, smem, s>>>(a, n_layers, n_tiles, mh, mw);
+  return cudaGetLastError();
+}
+
+template <int N>
+cudaError_t launch_k12_tcp_for_c(const RouteArgs& a, int n_layers, int router_blocks,
+                                 const CUtensorMap& mh, const CUtensorMap& mw, cudaStream_t s) {
+  if (a.c <= 4) return launch_k12_tcp<N, 4>(a, n_layers, router_blocks, mh, mw, s);
+  if (a.c <= 8) return launch_k12_tcp<N, 8>(a, n_layers, router_blocks, mh, mw, s);
+  if (a.c <= 16) return launch_k12_tcp<N, 16>(a, n_layers, router_blocks, mh, mw, s);
+  return launch_k12_tcp<N, 32>(a, n_layers, router_blocks, mh, mw, s);
+}
+
 template <int N>
 cudaError_t launch_k12_tc_for_c(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
                                 const CUtensorMap& mw, cudaStream_t s) {
@@ -109,5 +135,8 @@ cudaError_t launch_tc_n128(const RouteArgs& a, int n_layers, const CUtensorMap& 
                            const CUtensorMap& mw, cudaStream_t s);
 cudaError_t launch_tc_n256(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
                            const CUtensorMap& mw, cudaStream_t s);
+cudaError_t launch_tcp_n64(const RouteArgs& a, int n_layers, int router_blocks,
+                           const CUtensorMap& mh, const CUtensorMap& mw, cudaStream_t s);
+
 
 }  // namespace laser

@@ -71,6 +71,19 @@ bool make_map(CUtensorMap* m, const void* base, long long rows, int d, long long
             promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SMs of the current device (looked up once per device).
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 // Returns false if the tensor maps cannot be built for this call (the caller then uses the
 // warp-level router, which has no such requirement).
 bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, cudaError_t* err) {
@@ -89,6 +102,13 @@ bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, 
     return false;
   if (!make_map(&mw, a.wg, total_layers * a.E, a.d, a.ld_w, N, CU_TENSOR_MAP_L2_PROMOTION_L2_128B))
     return false;
+  // E <= 64: persistent router blocks, two per SM next to the selection blocks (the one-tile-
+  // per-block form stays reachable for the tests and for comparison; wider shapes have no room
+  // for two such blocks per SM)
+  if (N == 64 && g_test_router != LASER_TEST_ROUTER_TILE_ONESHOT) {
+    *err = launch_tcp_n64(a, n_layers, 2 * sm_count() - n_layers, mh, mw, s);
+    return true;
+  }
   if (N == 64) *err = launch_tc_n64(a, n_layers, mh, mw, s);
   else if (N == 128) *err = launch_tc_n128(a, n_layers, mh, mw, s);
   else *err = launch_tc_n256(a, n_layers, mh, mw, s);
@@ -110,7 +130,8 @@ cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
   // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block
   // (laser_test_set_router overrides the choice for the tests)
   bool few = (long long)n_layers * ((a.T + 127) / 128) * 4 <= 148;
-  if (g_test_router == LASER_TEST_ROUTER_TILE) few = false;
+  if (g_test_router == LASER_TEST_ROUTER_TILE || g_test_router == LASER_TEST_ROUTER_TILE_ONESHOT)
+    few = false;
   else if (g_test_router == LASER_TEST_ROUTER_SPLITK) few = true;
   if (few) return launch_k12_splitk_for_E(a, n_layers, s);
   if (E > 32) {
@@ -175,7 +196,7 @@ extern "C" int laser_version(void) { return 200; }
 
 extern "C" int laser_test_set_router(int mode) {
   if (mode != LASER_TEST_ROUTER_AUTO && mode != LASER_TEST_ROUTER_TILE &&
-      mode != LASER_TEST_ROUTER_SPLITK)
+      mode != LASER_TEST_ROUTER_SPLITK && mode != LASER_TEST_ROUTER_TILE_ONESHOT)
     return -1;
   const int prev = g_test_router;
   g_test_router = mode;

@@ -32,7 +32,7 @@ STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 DEV_LOAD_OVERFLOW = 1
 DEV_TIMEOUT = 2
 MAX_EXPERTS = 256
-ROUTER_AUTO, ROUTER_TILE, ROUTER_SPLITK = 0, 1, 2
+ROUTER_AUTO, ROUTER_TILE, ROUTER_SPLITK, ROUTER_TILE_ONESHOT = 0, 1, 2, 3
 
 EXPORTS = ("laser_version", "laser_strerror", "laser_workspace_bytes", "laser_route",
            "laser_route_layers", "laser_route_layers_profiled", "laser_host_arena_bytes",
