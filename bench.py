@@ -60,7 +60,7 @@ def workload_config(w, n_layers, n_copies=1):
             "cache": cache}
 
 
-DECODE_NODES_PER_CALL = 2   # a memset of the router's flags and one kernel
+DECODE_NODES_PER_CALL = 1   # calls of at most 112 tokens: one kernel (a thread-block cluster per layer)
 
 
 def launches_per_step(w, L) -> int:

@@ -71,6 +71,22 @@ template <int NT, int KU, int CMAX>
 __global__ void __launch_bounds__(kK2Threads)
 k12_route_select_splitk(const RouteArgs A, int n_layers) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
+  if (A.cluster_tiles > 0) {
+    // Few tiles per layer: the launch is one cluster per layer (rank 0 selects, ranks 1.. route
+    // one tile each).  The routers never wait, so every block reaches the cluster barrier, and
+    // the selection starts behind it with all records in place: no flags, no polling.
+    const int cs = A.cluster_tiles + 1;
+    const int rank = (int)blockIdx.x % cs, local_layer = (int)blockIdx.x / cs;
+    if (rank > 0) {
+      router_splitk_block<NT, KU>(A, local_layer, rank - 1, reinterpret_cast<float*>(dyn_smem));
+      __threadfence();
+    }
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (rank == 0)
+      k2_block<CMAX, (NT * 8 <= 32)>(A, A.layer0 + local_layer, dyn_smem, nullptr, 16);
+    return;
+  }
   if ((int)blockIdx.x < n_layers) {
     const int layer = A.layer0 + blockIdx.x;
     const int* ready = reinterpret_cast<const int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);

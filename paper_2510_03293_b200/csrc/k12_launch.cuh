@@ -101,6 +101,22 @@ cudaError_t launch_k12_splitk(const RouteArgs& a, int n_layers, cudaStream_t s) 
     if (e != cudaSuccess) return e;
   }
   const unsigned tiles = (unsigned)((a.T + 15) / 16);
+  if (a.cluster_tiles > 0) {
+    // one cluster per layer: the selection block and the layer's router tiles
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_layers * (1 + tiles));
+    cfg.blockDim = dim3(kK2Threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1 + tiles;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k12_route_select_splitk<NT, KU, CMAX>, a, n_layers);
+  }
   k12_route_select_splitk<NT, KU, CMAX>
       <<<n_layers * (1 + tiles), kK2Threads, smem, s>>>(a, n_layers);
   return cudaGetLastError();

@@ -411,10 +411,14 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   // A wait that runs out (or a router tile that gave up) aborts the layer: the status bit is
   // raised and the layer's abort word set, after which neither this block nor the dispatch
   // reads the layer's scratch records again (they may be unwritten).
-  int* abort_word = const_cast<int*>(ready) + abort_word_index(T);
+  // (the layer's control words live behind its ready flags; without flags -- the records are
+  // all there when the block starts -- nothing cleared them, so this block does)
+  int* ctrl = reinterpret_cast<int*>(A.ws + (size_t)layer * A.ws_ls + A.lay.ready);
+  int* abort_word = ctrl + abort_word_index(T);
+  if (!ready && tid == 0) *abort_word = 0;
   auto give_up = [&]() {
     if (A.status) atomicOr(A.status, 2);
-    if (ready) st_release(abort_word, 1);
+    st_release(abort_word, 1);
     s_gave_up = 1;
   };
   int too_big = 0;
@@ -428,6 +432,8 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
     if (v < 0 || v > kK2FastMaxLoad - T) too_big = 1;
   }
   const bool wide = __syncthreads_or(too_big) || !k2_fast_shape(k, c);
+  // how the decision tokens' choices are left for the dispatch: rank masks (1) or rank lists (0)
+  if (tid == 0) ctrl[mode_word_index(T)] = (!wide && !SMALL && chain) ? 1 : 0;
 
   if (wide) {
     if (warp == 0) {
@@ -452,7 +458,6 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
       if (!ok && lane == 0) give_up();
     }
   } else if (!SMALL && chain) {
-    if (tid == 0 && ready) const_cast<int*>(ready)[mode_word_index(T)] = 1;   // choices as masks
     k2_chain_layer<CMAX>(A, layer, chain_smem, sm.L, sm.Lin, &s_gave_up, ready, router_rows,
                          give_up);
   } else {

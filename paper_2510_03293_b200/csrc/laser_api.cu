@@ -125,15 +125,28 @@ cudaError_t launch_k12_splitk_for_E(const RouteArgs& a, int n_layers, cudaStream
   return launch_splitk_e256(a, n_layers, s);
 }
 
-cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
-  const int E = a.E;
-  // few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block
-  // (laser_test_set_router overrides the choice for the tests)
+// few tokens: 128-token tiles would leave most SMs idle, so route 16 tokens per block
+// (laser_test_set_router overrides the choice for the tests)
+bool use_splitk(const RouteArgs& a, int n_layers) {
   bool few = (long long)n_layers * ((a.T + 127) / 128) * 4 <= 148;
   if (g_test_router == LASER_TEST_ROUTER_TILE || g_test_router == LASER_TEST_ROUTER_TILE_ONESHOT)
     few = false;
   else if (g_test_router == LASER_TEST_ROUTER_SPLITK) few = true;
-  if (few) return launch_k12_splitk_for_E(a, n_layers, s);
+  return few;
+}
+
+// Calls of at most 7 router tiles per layer (112 tokens) whose dispatch runs inside the selection
+// block are launched as one thread-block cluster per layer: no ready flags, so no memset.
+int cluster_tiles_for(const RouteArgs& a, int n_layers) {
+  const int tiles = (a.T + 15) / 16;
+  if (!use_splitk(a, n_layers) || tiles > 7 || !a.fuse_dispatch || g_test_withhold_tile >= 0)
+    return 0;
+  return tiles;
+}
+
+cudaError_t launch_k12_for_E(const RouteArgs& a, int n_layers, cudaStream_t s) {
+  const int E = a.E;
+  if (use_splitk(a, n_layers)) return launch_k12_splitk_for_E(a, n_layers, s);
   if (E > 32) {
     cudaError_t err = cudaSuccess;
     if (launch_k12_tensor_memory(a, n_layers, s, &err)) return err;
@@ -169,8 +182,10 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   }
   // clear the router's ready flags of these layers (one strided memset), then one launch for
   // the router and the ordered selection, one for the dispatch
+  a.cluster_tiles = cluster_tiles_for(a, n);
   const size_t ready_bytes = sizeof(int32_t) * (size_t)((a.T + 15) / 16 + 2);
-  if (cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
+  if (a.cluster_tiles == 0 &&
+      cudaMemset2DAsync(a.ws + (size_t)layer0 * a.ws_ls + a.lay.ready, a.ws_ls, 0, ready_bytes,
                         (size_t)n, s) != cudaSuccess)
     return LASER_ERR_CUDA;
   if (!mark(1)) return LASER_ERR_CUDA;

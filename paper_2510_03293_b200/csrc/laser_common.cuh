@@ -77,6 +77,9 @@ struct RouteArgs {
   int fuse_dispatch;       // 1 = the selection block also runs the dispatch of its layer (calls
                            //     of a few groups), and no dispatch kernel is launched
   int layer0;              // first layer of this launch
+  int cluster_tiles;       // > 0: the layer's router tiles and its selection block form one
+                           //      thread-block cluster (that many tiles + 1) and meet at the
+                           //      cluster barrier; no ready flags are used.  0: ready flags
   long long wait_cycles;   // limit of the selection's waits for the router, in clock cycles
   int withhold_tile;       // test hook: the router tile with this index publishes no flag (-1: none)
   float eps_high[kMaxLayersPerLaunch];

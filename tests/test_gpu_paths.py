@@ -117,3 +117,41 @@ def test_a_wait_that_runs_out_sets_the_timeout_bit(cuda_device, force_router, ro
     assert 0 <= int(g["loads"].sum()) <= T * k and int(g["loads"].min()) >= 0
     g = run_gpu(cuda_device, hb, wb, bias, z, k, c, 0.5, 0.5)
     check_against_oracle(g, hb, wb, bias, z, k, c, 0.5, 0.5)
+
+
+@pytest.mark.parametrize("T,d,E,k,c", [(100, 256, 64, 6, 8), (112, 128, 256, 8, 16),
+                                       (17, 64, 100, 5, 20), (64, 2048, 64, 6, 8),
+                                       (1, 256, 64, 6, 8), (97, 512, 8, 2, 4)])
+def test_calls_of_a_few_tiles_run_as_one_cluster_per_layer(cuda_device, T, d, E, k, c):
+    """At most 112 tokens: the layer's router tiles and its selection block are launched as one
+    thread-block cluster and meet at the cluster barrier instead of ready flags.  Several
+    layers at once must equal the layers routed one by one, and each the oracle."""
+    import torch
+
+    from paper_2510_03293_b200 import laser
+    from gpu_util import to_dev_bf16
+
+    dev = cuda_device
+    L = 5
+    layers = [layer(T, d, E, seed=700 + l + T) for l in range(L)]
+    hb = np.stack([x[0] for x in layers]); wb = np.stack([x[1] for x in layers])
+    bias = np.stack([x[2] for x in layers])
+    rng = np.random.default_rng(T + E)
+    loads0 = rng.integers(0, 4, (L, E)).astype(np.int32)
+    p = laser.make_params(T, d, E, k, c, 0.5, 0.5, 1, 4)
+    loads = torch.from_numpy(loads0.copy()).to(dev)
+    bins = torch.zeros((L, 4), dtype=torch.int32, device=dev)
+    # a workspace full of ones: nothing clears it for this kind of call, and nothing has to
+    ws = torch.full((laser.workspace_bytes(p) * L,), 0x5A, dtype=torch.uint8, device=dev)
+    r = laser.route_layers(to_dev_bf16(hb, dev), to_dev_bf16(wb, dev),
+                           torch.from_numpy(bias).to(dev), loads, p, bin_loads=bins,
+                           want_logits=True, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    for l in range(L):
+        g = dict(expert_ids=r.expert_ids[l].cpu().numpy(), weights=r.weights[l].cpu().numpy(),
+                 offsets=r.offsets[l].cpu().numpy(), perm=r.perm[l].cpu().numpy(),
+                 loads=loads[l].cpu().numpy(), bin_loads=bins[l].cpu().numpy(),
+                 logits=r.logits[l].cpu().numpy(), status=0)
+        check_against_oracle(g, hb[l], wb[l], bias[l], loads0[l], k, c, 0.5, 0.5, 1, 4,
+                             bins0=np.zeros(4, np.int32))
