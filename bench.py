@@ -100,7 +100,10 @@ def recorded_traffic(workload: str, tokens: int):
 def router_kernel_name(w, L) -> str:
     if L * ((w.T + 127) // 128) * 4 <= 148:
         return "k12_route_select_splitk (split-K contraction + score epilogue + ordered selection)"
-    if w.E > 32:
+    if 32 < w.E <= 64:
+        return ("k12_route_select_tcp (persistent tcgen05 contraction + score epilogue + ordered "
+                "selection)")
+    if w.E > 64:
         return "k12_route_select_tc (tcgen05 contraction + score epilogue + ordered selection)"
     return "k12_route_select (mma.sync contraction + score epilogue + ordered selection)"
 

@@ -17,7 +17,8 @@ def force_router():
     from paper_2510_03293_b200 import laser
 
     def choose(name):
-        laser.test_set_router({"tile": laser.ROUTER_TILE, "splitk": laser.ROUTER_SPLITK}[name])
+        laser.test_set_router({"tile": laser.ROUTER_TILE, "splitk": laser.ROUTER_SPLITK,
+                               "oneshot": laser.ROUTER_TILE_ONESHOT}[name])
 
     yield choose
     laser.test_set_router(laser.ROUTER_AUTO)
@@ -69,6 +70,19 @@ def test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B):
     if T >= 100 and d >= 1024 and 0 < eps < 1 and c > k:
         frac = float((ref["cstar"] > 0).mean())
         assert 0.005 < frac < 0.995, f"only one branch exercised (expanded fraction {frac})"
+
+
+@pytest.mark.parametrize("T,d,E,k,c,eps,tfix,renorm,B", [
+    (1000, 2048, 64, 6, 8, 0.40, 0.80, 0, 8), (515, 512, 64, 6, 10, 0.30, 0.50, 1, 8),
+    (4900, 512, 64, 6, 8, 0.40, 0.80, 0, 8), (700, 264, 48, 4, 12, 0.5, 0.4, 1, 6),
+    (130, 256, 33, 3, 5, 0.5, 0.5, 1, 3), (40000, 128, 64, 6, 8, 0.5, 0.6, 1, 8)])
+@pytest.mark.parametrize("router", ["tile", "oneshot"])
+def test_both_forms_of_the_64_column_router(cuda_device, force_router, router, T, d, E, k, c, eps,
+                                            tfix, renorm, B):
+    """32 < E <= 64 has a persistent router (several tiles per block, more tiles than blocks in
+    the last case) and a one-tile-per-block form; both must equal the oracle."""
+    force_router(router)
+    test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B)
 
 
 @pytest.mark.parametrize("T,d,E,k,c,eps,tfix,renorm,B", [c_ for c_ in CASES if c_[0] < 4000])
