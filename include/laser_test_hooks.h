@@ -17,7 +17,7 @@ enum {
   LASER_TEST_ROUTER_AUTO = 0,
   LASER_TEST_ROUTER_TILE = 1,          /* the 128-token-tile routers */
   LASER_TEST_ROUTER_SPLITK = 2,        /* the 16-token split-K router */
-  LASER_TEST_ROUTER_TILE_ONESHOT = 3   /* as TILE, but 32 < E <= 64 takes the one-tile-per-block
+  LASER_TEST_ROUTER_TILE_ONESHOT = 3   /* as TILE, but every E > 32 takes the one-tile-per-block
                                           form of the tensor-memory router, not the persistent one */
 };
 

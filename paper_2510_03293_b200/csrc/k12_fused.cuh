@@ -140,11 +140,11 @@ k12_route_select_tc(const RouteArgs A, int n_layers, const __grid_constant__ CUt
   }
 }
 
-// The persistent form of the tensor-memory router (E <= 128): the first n_layers blocks select,
+// The persistent form of the tensor-memory router (E <= 64, or 128 < E <= 256 with c <= 16): the first n_layers blocks select,
 // every other block walks the tiles b, b + P, ... of all layers (tile id = tile index * n_layers
 // + layer).
 template <int N, int CMAX>
-__global__ void __launch_bounds__(kK2Threads, 2)
+__global__ void __launch_bounds__(kK2Threads, N <= 64 ? 2 : 1)
 k12_route_select_tcp(const RouteArgs A, int n_layers, int n_tiles,
                      const __grid_constant__ CUtensorMap map_h,
                      const __grid_constant__ CUtensorMap map_w) {

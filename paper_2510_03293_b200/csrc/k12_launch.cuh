@@ -54,7 +54,7 @@ cudaError_t launch_k12_tc(const RouteArgs& a, int n_layers, const CUtensorMap& m
   return cudaGetLastError();
 }
 
-// Persistent form (N <= 128): router_blocks blocks walk all tiles of the launch.
+// Persistent form (N = 64 or 256): router_blocks blocks walk all tiles of the launch.
 template <int N, int CMAX>
 cudaError_t launch_k12_tcp(const RouteArgs& a, int n_layers, int router_blocks,
                            const CUtensorMap& mh, const CUtensorMap& mw, cudaStream_t s) {
@@ -151,6 +151,8 @@ cudaError_t launch_tc_n128(const RouteArgs& a, int n_layers, const CUtensorMap& 
                            const CUtensorMap& mw, cudaStream_t s);
 cudaError_t launch_tc_n256(const RouteArgs& a, int n_layers, const CUtensorMap& mh,
                            const CUtensorMap& mw, cudaStream_t s);
+cudaError_t launch_tcp_n256(const RouteArgs& a, int n_layers, int router_blocks,
+                            const CUtensorMap& mh, const CUtensorMap& mw, cudaStream_t s);
 cudaError_t launch_tcp_n64(const RouteArgs& a, int n_layers, int router_blocks,
                            const CUtensorMap& mh, const CUtensorMap& mw, cudaStream_t s);
 

@@ -20,9 +20,12 @@
 namespace laser {
 
 template <int N>
-__host__ __device__ constexpr int tcp_stages() { return N <= 64 ? 3 : 2; }
+__host__ __device__ constexpr int tcp_stages() { return N <= 64 ? 3 : (N == 256 ? 4 : 2); }
 template <int N>
-__host__ __device__ constexpr size_t tcp_tile_bytes() { return (size_t)kTcTileM * (N + 1) * 4; }
+__host__ __device__ constexpr size_t tcp_tile_bytes() {
+  // N = 256 scores from tensor memory and keeps only a 32-float row per thread of the team
+  return N == 256 ? (size_t)4 * 32 * 33 * 4 : (size_t)kTcTileM * (N + 1) * 4;
+}
 // stages (1024-byte aligned, hence the slack) + logits rows + bias + barriers
 template <int N>
 __host__ __device__ constexpr size_t tcp_smem_bytes() {
@@ -116,6 +119,10 @@ __device__ __forceinline__ void router_tcp_team(const RouteArgs& A, int n_layers
     if (tid == 0 && rt != A.withhold_tile) { __threadfence(); st_release(ready + rt, 1); }
   }
 }
+
+}  // namespace laser
+#include "k1_router_tcp256.cuh"
+namespace laser {
 
 // Router role of one persistent block (256 threads): tiles first, first + step, ... < n_tiles of
 // the launch's n_layers layers.  N: accumulator columns (64; 128 compiles but two such blocks do
@@ -223,8 +230,12 @@ __device__ __forceinline__ void router_tcp_block(const RouteArgs& A, const CUten
     }
   } else {
     // ---- scoring team (see the second half of this function)
-    router_tcp_team<N, CL>(A, n_layers, first, step, n_tiles, tmem, tile, bias_s, s_fm, acc_full,
-                           acc_empty, abort);
+    if constexpr (N == 256)
+      router_tcp256_team(A, n_layers, first, step, n_tiles, tmem, tile, bias_s, s_fm, acc_full,
+                         acc_empty, abort);
+    else
+      router_tcp_team<N, CL>(A, n_layers, first, step, n_tiles, tmem, tile, bias_s, s_fm, acc_full,
+                             acc_empty, abort);
   }
   __syncwarp();
   tc_fence_before();

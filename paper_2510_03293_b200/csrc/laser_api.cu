@@ -109,6 +109,14 @@ bool launch_k12_tensor_memory(const RouteArgs& a, int n_layers, cudaStream_t s, 
     *err = launch_tcp_n64(a, n_layers, 2 * sm_count() - n_layers, mh, mw, s);
     return true;
   }
+  // 128 < E <= 256 with lists of at most 16: one persistent block per SM (four 48 KB stages, two
+  // accumulators fill the tensor memory); the selection blocks take an SM each
+  if (N == 256 && a.c <= 16 && !a.trim_random && g_test_router != LASER_TEST_ROUTER_TILE_ONESHOT) {
+    int blocks = sm_count() - n_layers;
+    if (blocks < sm_count() / 2) blocks = sm_count() / 2;
+    *err = launch_tcp_n256(a, n_layers, blocks, mh, mw, s);
+    return true;
+  }
   if (N == 64) *err = launch_tc_n64(a, n_layers, mh, mw, s);
   else if (N == 128) *err = launch_tc_n128(a, n_layers, mh, mw, s);
   else *err = launch_tc_n256(a, n_layers, mh, mw, s);

@@ -75,12 +75,15 @@ def test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B):
 @pytest.mark.parametrize("T,d,E,k,c,eps,tfix,renorm,B", [
     (1000, 2048, 64, 6, 8, 0.40, 0.80, 0, 8), (515, 512, 64, 6, 10, 0.30, 0.50, 1, 8),
     (4900, 512, 64, 6, 8, 0.40, 0.80, 0, 8), (700, 264, 48, 4, 12, 0.5, 0.4, 1, 6),
-    (130, 256, 33, 3, 5, 0.5, 0.5, 1, 3), (40000, 128, 64, 6, 8, 0.5, 0.6, 1, 8)])
+    (130, 256, 33, 3, 5, 0.5, 0.5, 1, 3), (40000, 128, 64, 6, 8, 0.5, 0.6, 1, 8),
+    (777, 1024, 256, 8, 16, 0.30, 0.25, 1, 32), (1500, 264, 200, 8, 12, 0.3, 0.25, 0, 8),
+    (300, 128, 129, 4, 4, 0.5, 0.5, 1, 3), (40000, 64, 256, 8, 16, 0.4, 0.3, 1, 16)])
 @pytest.mark.parametrize("router", ["tile", "oneshot"])
-def test_both_forms_of_the_64_column_router(cuda_device, force_router, router, T, d, E, k, c, eps,
+def test_both_forms_of_the_tensor_memory_router(cuda_device, force_router, router, T, d, E, k, c, eps,
                                             tfix, renorm, B):
-    """32 < E <= 64 has a persistent router (several tiles per block, more tiles than blocks in
-    the last case) and a one-tile-per-block form; both must equal the oracle."""
+    """32 < E <= 64, and 128 < E <= 256 with lists of at most 16, have a persistent router
+    (several tiles per block, more tiles than blocks in the cases of 40000 tokens) and a
+    one-tile-per-block form; both must equal the oracle."""
     force_router(router)
     test_route_matches_oracle(cuda_device, T, d, E, k, c, eps, tfix, renorm, B)
 

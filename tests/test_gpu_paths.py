@@ -18,7 +18,8 @@ def force_router():
     from paper_2510_03293_b200 import laser
 
     def choose(name):
-        laser.test_set_router({"tile": laser.ROUTER_TILE, "splitk": laser.ROUTER_SPLITK}[name])
+        laser.test_set_router({"tile": laser.ROUTER_TILE, "splitk": laser.ROUTER_SPLITK,
+                               "oneshot": laser.ROUTER_TILE_ONESHOT}[name])
 
     yield choose
     laser.test_set_router(laser.ROUTER_AUTO)
@@ -92,7 +93,9 @@ def test_loads_beyond_the_packed_key_range(cuda_device, force_router, router, T,
 
 @pytest.mark.parametrize("router,T,d,E,k,c,tile", [
     ("tile", 1000, 256, 8, 2, 4, 1),       # warp-level router, 128-token tiles
-    ("tile", 1000, 256, 64, 6, 8, 2),      # tensor-memory router
+    ("tile", 1000, 256, 64, 6, 8, 2),      # tensor-memory router, persistent blocks
+    ("tile", 1000, 256, 256, 8, 16, 3),    # ... with 256 accumulator columns
+    ("oneshot", 1000, 256, 64, 6, 8, 2),   # ... one tile per block
     ("splitk", 300, 256, 64, 6, 8, 5),     # split-K router, 16-token tiles, fused dispatch off
     ("splitk", 200, 256, 64, 6, 8, 3),     # ... dispatch inside the selection block
     ("tile", 700, 128, 256, 8, 40, 0),     # one-warp scan (candidate lists wider than a warp)
