@@ -285,8 +285,9 @@ def run_layers(args, w, ctx, full):
     p = laser.make_params(w.T, w.d, w.E, w.k, w.c, w.eps_high[0], w.t_fix, w.renormalize, w.n_bins,
                           update_granularity=args.granularity,
                           trim_mode=0 if args.random_trim is None else 1,
-                          seed=args.random_trim or 0)
-    # load counters of experts and bins in one buffer, so that a step resets them with one memset
+                          seed=args.random_trim or 0, fresh_loads=1)
+    # every step starts from empty load counters (the method resets the loads per batch): the
+    # call itself does that (fresh_loads), no memset between steps
     state = torch.zeros((L * (w.E + w.n_bins),), dtype=torch.int32, device=dev)
     loads = state[:L * w.E].view(L, w.E)
     bins = state[L * w.E:].view(L, w.n_bins)
@@ -314,7 +315,6 @@ def run_layers(args, w, ctx, full):
 
     def step(events=None, eps=None):
         nonlocal out, it
-        state.zero_()
         out = laser.route_layers(hiddens[it % n_copies], data["w_g"], data["bias"], loads, p,
                                  bin_loads=bins, eps_high=data["eps_high"] if eps is None else eps,
                                  t_fix=data["t_fix"], out=out, workspace=ws, stage_events=events)

@@ -98,6 +98,11 @@ typedef struct laser_params {
   int32_t update_granularity;
   int32_t renormalize;
   int32_t n_bins;
+  int32_t fresh_loads; /* 0: loads and bin_loads are in/out and the call adds to them.
+                          1: the call starts from empty counters (the method resets the loads at
+                          the start of a batch): what loads and bin_loads hold on entry is ignored
+                          and they return this call's counts.  (This word was padding before:
+                          a zeroed structure keeps the old behaviour.) */
   int64_t ld_hidden, ld_w;
   uint64_t seed; /* RANDOM trimming: generator key */
 } laser_params;

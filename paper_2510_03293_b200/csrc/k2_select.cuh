@@ -423,7 +423,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
   };
   int too_big = 0;
   for (int e = tid; e < E; e += kK2Threads) {
-    const int32_t v = g_loads[e];
+    const int32_t v = A.fresh ? 0 : g_loads[e];
     sm.L[e] = v;
     sm.Lin[e] = v;
     sm.Lvis[e] = v;
@@ -573,7 +573,7 @@ __device__ __forceinline__ void k2_block(const RouteArgs& A, int layer, unsigned
         const int be = A.e2b ? A.e2b[e] : e / per;
         if (be == b) s += s_cnt[e];
       }
-      bl[b] += s;
+      bl[b] = (A.fresh ? 0 : bl[b]) + s;
     }
   }
   if (A.fuse_dispatch && !s_gave_up) {   // (s_gave_up was written before the barriers above)

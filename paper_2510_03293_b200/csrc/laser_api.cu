@@ -182,9 +182,17 @@ int enqueue_group(RouteArgs& a, int layer0, int n, const laser_params* p, const 
   a.wait_cycles = g_test_withhold_tile >= 0 ? g_test_wait_cycles : kK2WaitCycles;
   if (!mark(0)) return LASER_ERR_CUDA;
   if (a.T == 0) {
-    // nothing to route: the call's offsets are all zero, loads and bins stay as they are
+    // nothing to route: the call's offsets are all zero, loads and bins stay as they are (or
+    // are this call's counts: zero)
     if (cudaMemsetAsync(a.offsets + (size_t)layer0 * (a.E + 1), 0,
                         sizeof(int32_t) * (size_t)n * (a.E + 1), s) != cudaSuccess)
+      return LASER_ERR_CUDA;
+    if (a.fresh &&
+        (cudaMemsetAsync(a.loads + (size_t)layer0 * a.E, 0, sizeof(int32_t) * (size_t)n * a.E,
+                         s) != cudaSuccess ||
+         (a.bin_loads &&
+          cudaMemsetAsync(a.bin_loads + (size_t)layer0 * a.n_bins, 0,
+                          sizeof(int32_t) * (size_t)n * a.n_bins, s) != cudaSuccess)))
       return LASER_ERR_CUDA;
     return (mark(1) && mark(2) && mark(3)) ? LASER_OK : LASER_ERR_CUDA;
   }
@@ -349,6 +357,7 @@ extern "C" int laser_route_layers_profiled(
   a.loads = loads;
   a.e2b = expert_to_bin;
   a.bin_loads = bin_loads;
+  a.fresh = p->fresh_loads != 0;
   a.expert_ids = expert_ids;
   a.weights = weights;
   a.offsets = offsets;

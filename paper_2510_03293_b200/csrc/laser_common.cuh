@@ -59,6 +59,7 @@ struct RouteArgs {
   int32_t* loads;          // [L, E]
   const int32_t* e2b;      // [E] or null
   int32_t* bin_loads;      // [L, B] or null
+  int fresh;               // the counters start from zero whatever loads / bin_loads hold
   int32_t* expert_ids;     // [L, T, k]
   float* weights;          // [L, T, k]
   int32_t* offsets;        // [L, E+1]

@@ -48,6 +48,7 @@ class LaserParams(ctypes.Structure):
                 ("eps_high", ctypes.c_float), ("t_fix", ctypes.c_float),
                 ("trim_mode", ctypes.c_int32), ("update_granularity", ctypes.c_int32),
                 ("renormalize", ctypes.c_int32), ("n_bins", ctypes.c_int32),
+                ("fresh_loads", ctypes.c_int32),
                 ("ld_hidden", ctypes.c_int64), ("ld_w", ctypes.c_int64),
                 ("seed", ctypes.c_uint64)]
 
@@ -138,9 +139,11 @@ def strerror(status: int) -> str:
 
 
 def make_params(T, d, E, k, c, eps_high, t_fix, renormalize=1, n_bins=1, ld_hidden=None,
-                ld_w=None, trim_mode=0, update_granularity=1, seed=0) -> LaserParams:
+                ld_w=None, trim_mode=0, update_granularity=1, seed=0,
+                fresh_loads=0) -> LaserParams:
     return LaserParams(T, d, E, k, c, eps_high, t_fix, trim_mode, update_granularity,
-                       int(renormalize), n_bins, d if ld_hidden is None else ld_hidden,
+                       int(renormalize), n_bins, int(fresh_loads),
+                       d if ld_hidden is None else ld_hidden,
                        d if ld_w is None else ld_w, seed)
 
 

@@ -37,7 +37,7 @@ class Padded:
 
 
 def run_gpu(dev, hb, wb, bias, loads0, k, c, eps, tfix, renorm=1, n_bins=1, e2b=None,
-            bins0=None, want_logits=True, skew=0):
+            bins0=None, want_logits=True, skew=0, fresh=0):
     """One laser_route call; returns dict of numpy outputs.  Checks the canaries."""
     import torch
 
@@ -45,7 +45,7 @@ def run_gpu(dev, hb, wb, bias, loads0, k, c, eps, tfix, renorm=1, n_bins=1, e2b=
 
     T, d = hb.shape
     E = wb.shape[0]
-    p = laser.make_params(T, d, E, k, c, eps, tfix, renorm, n_bins)
+    p = laser.make_params(T, d, E, k, c, eps, tfix, renorm, n_bins, fresh_loads=fresh)
     hidden = to_dev_bf16(hb, dev) if T > 0 else torch.empty((0, d), dtype=torch.bfloat16, device=dev)
     wg = to_dev_bf16(wb, dev)
     loads = torch.from_numpy(np.asarray(loads0, np.int32).copy()).to(dev)

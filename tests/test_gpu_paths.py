@@ -158,3 +158,22 @@ def test_calls_of_a_few_tiles_run_as_one_cluster_per_layer(cuda_device, T, d, E,
                  logits=r.logits[l].cpu().numpy(), status=0)
         check_against_oracle(g, hb[l], wb[l], bias[l], loads0[l], k, c, 0.5, 0.5, 1, 4,
                              bins0=np.zeros(4, np.int32))
+
+
+@pytest.mark.parametrize("router", ROUTERS)
+@pytest.mark.parametrize("T,d,E,k,c", [(0, 64, 8, 2, 4), (90, 128, 64, 6, 8), (700, 256, 8, 2, 4),
+                                       (900, 128, 64, 6, 8), (600, 128, 256, 8, 16),
+                                       (300, 128, 256, 8, 40)])
+def test_a_call_that_starts_from_empty_counters(cuda_device, force_router, router, T, d, E, k, c):
+    """fresh_loads = 1: whatever the load and bin counters hold on entry is ignored; the call
+    equals the oracle started from zero loads, and the counters return the call's own counts."""
+    force_router(router)
+    hb, wb, bias = layer(T, d, E, seed=T + E + 5)
+    rng = np.random.default_rng(T + c)
+    junk_loads = rng.integers(-5, 1 << 28, E).astype(np.int32)
+    junk_bins = rng.integers(-5, 1 << 28, 4).astype(np.int32)
+    g = run_gpu(cuda_device, hb, wb, bias, junk_loads, k, c, 0.5, 0.5, 1, 4, bins0=junk_bins,
+                fresh=1)
+    zero_l, zero_b = np.zeros(E, np.int32), np.zeros(4, np.int32)
+    check_against_oracle(g, hb, wb, bias, zero_l, k, c, 0.5, 0.5, 1, 4, bins0=zero_b)
+    assert int(g["loads"].sum()) == T * k and int(g["bin_loads"].sum()) == T * k
