@@ -228,7 +228,7 @@ def route_layers(hidden, w_g, bias, loads, p: LaserParams, *, expert_to_bin=None
     s = torch.cuda.current_stream(dev) if stream is None else stream
     ev_p = None
     if stage_events is not None:
-        ev_arr = (_vp * 4)(*[int(e.cuda_event) for e in stage_events])
+        ev_arr = (_vp * 4)(*[None if e is None else int(e.cuda_event) for e in stage_events])
         ev_p = ctypes.cast(ev_arr, _vp)
     rc = _lib.laser_route_layers_profiled(
         L, _ptr(hidden), _ptr(w_g), _ptr(bias), _ptr(loads), _ptr(expert_to_bin),
