@@ -177,3 +177,27 @@ def test_a_call_that_starts_from_empty_counters(cuda_device, force_router, route
     zero_l, zero_b = np.zeros(E, np.int32), np.zeros(4, np.int32)
     check_against_oracle(g, hb, wb, bias, zero_l, k, c, 0.5, 0.5, 1, 4, bins0=zero_b)
     assert int(g["loads"].sum()) == T * k and int(g["bin_loads"].sum()) == T * k
+
+
+def bf16_bits(x):
+    """bf16 bit patterns of values that are exactly representable (small integers, halves)."""
+    return (np.asarray(x, np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+@pytest.mark.parametrize("router", ROUTERS + ["oneshot"])
+@pytest.mark.parametrize("T,d,E,k,c", [(500, 64, 64, 6, 8), (700, 32, 256, 8, 16),
+                                       (300, 64, 128, 4, 12), (400, 48, 8, 2, 4)])
+def test_rows_with_many_equal_logits(cuda_device, force_router, router, T, d, E, k, c):
+    """Hidden states and gate weights from {-1, 0, 1}: logits are small integers, most of them
+    shared by several experts of a row, so rankings are decided by the index inside groups of
+    equal logits next to groups that differ (the sorting-network epilogues have to notice)."""
+    force_router(router)
+    rng = np.random.default_rng(T + E)
+    hb = bf16_bits(rng.integers(-1, 2, (T, d)))
+    wb = bf16_bits(rng.integers(-1, 2, (E, d)))
+    bias = (rng.integers(0, 3, E) * 0.5).astype(np.float32)
+    loads0 = rng.integers(0, 3, E).astype(np.int32)
+    g = run_gpu(cuda_device, hb, wb, bias, loads0, k, c, 0.9, 0.2, 1, 4,
+                bins0=np.zeros(4, np.int32))
+    check_against_oracle(g, hb, wb, bias, loads0, k, c, 0.9, 0.2, 1, 4,
+                         bins0=np.zeros(4, np.int32))
