@@ -262,6 +262,8 @@ def _route_layers_strided(dev, hb, wb, bias, ld_h, ld_w, k, c, eps, tfix, B):
     (2, 333, 520, 100, 5, 12, 528, 536),    # ... with padded rows and 128 accumulator columns
     (2, 150, 256, 256, 8, 16, 320, 256),    # ... 256 accumulator columns, two-pass epilogue
     (3, 300, 264, 8, 2, 4, 272, 280),       # warp-level router with padded rows
+    (8, 4100, 128, 256, 8, 16, 128, 128),   # persistent routers: more tiles than blocks, tiles of
+    (11, 5000, 64, 64, 6, 8, 64, 64),       # different layers one after the other in a block
 ])
 def test_batched_layers_ragged_tiles_and_row_pitch(cuda_device, force_router, router, L, T, d, E,
                                                    k, c, ld_h, ld_w):
